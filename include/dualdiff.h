@@ -1,0 +1,153 @@
+/*
+ * dualdiff.h -- C ABI of the B200 (sm_100a) library for the data-parallel core
+ * of one DualDiffusion verification step (speculative decoding for masked
+ * diffusion language models):
+ *
+ *   dd_bidir_attention : full-sequence bidirectional multi-head attention, the
+ *                        O(L^2)-per-step cost of Section 2.2 (Eq. 3 evaluated
+ *                        over the whole key range, no causal mask, no cache).
+ *   dd_verify          : the verification algorithm A(p_D, p_V, x^D) of
+ *                        Algorithm 1 / Section 3.2: Trust Verifier (Eq. 4),
+ *                        KL-divergence remasking (Eq. 5, Eq. 6) and
+ *                        confidence remasking (Eq. 7).
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named without a prefix are DEVICE pointers owned by the caller;
+ *     the *_host entry points take HOST pointers (pinned memory if the copies
+ *     are to be asynchronous).  Tensors are contiguous, innermost dimension
+ *     last.  bf16 tensors are passed as void* to raw bf16 storage.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All work is enqueued on it; no entry point synchronises the stream.
+ *   - The return value is a dd_status; 0 is success.  On any error nothing is
+ *     launched and no output is written.  The library never falls back to a
+ *     CPU computation.
+ *   - The library keeps a small per-device scratch area (partial results and
+ *     completion counters of dd_verify, staging buffers of the *_host calls).
+ *     It is allocated with cudaMalloc the first time a call on that device
+ *     needs it, or needs more than before, which synchronises the device: make
+ *     one call of the intended size before relying on asynchrony.  Two calls
+ *     that may run concurrently on the same device (different streams, no
+ *     ordering between them) would share this scratch and are not supported.
+ *     dd_release() frees it.
+ */
+#ifndef DUALDIFF_H_
+#define DUALDIFF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DD_OK = 0,
+    DD_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, unknown mode, NaN tau, k < 0 */
+    DD_ERR_UNSUPPORTED = -2, /* valid request outside what the kernels implement          */
+    DD_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed; see dd_last_cuda_error  */
+    DD_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see dd_attention_status) */
+} dd_status;
+
+/* `mode` argument of dd_verify: algorithm in the low 8 bits, flag bits above. */
+enum {
+    DD_MODE_TRUST = 0,             /* Eq. 4: nothing is remasked                              */
+    DD_MODE_KL = 1,                /* Eq. 5 score; remask if KL > tau (threshold rule)        */
+    DD_MODE_CONF = 2,              /* Eq. 7 score; remask if c_V < tau (threshold rule)       */
+    DD_FLAG_PROBABILISTIC = 0x100, /* KL: remask w.p. Eq. 6; CONF: remask w.p. 1 - c_V        */
+    DD_FLAG_EMIT_DRAFTER = 0x200   /* kept positions keep tokens[i] instead of the verifier's
+                                      most likely token (Eq. 4 taken literally)               */
+};
+
+/*
+ * Bidirectional attention (Section 2.2; Eq. 3 with the key range 1..L):
+ *     out[b,h,i,:] = sum_j softmax_j(scale * q[b,h,i,:] . k[b,h,j,:]) v[b,h,j,:],
+ * j over all N positions.  q, k, v, out: [B,H,N,D] bf16, D innermost, 16-byte
+ * aligned, out not overlapping the inputs.  Scores and the softmax are
+ * accumulated in fp32; the result is rounded to bf16 once.
+ * Supported: D in {64,128}; any N >= 1; B*H*ceil(N/128) < 2^31.
+ * Errors: DD_ERR_INVALID_ARG (null pointer, B/H/N/D <= 0, scale not finite),
+ * DD_ERR_UNSUPPORTED (other D, misaligned pointer), DD_ERR_CUDA.
+ */
+int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
+                       int B, int H, int N, int D, float scale, void *stream);
+
+/*
+ * Verification algorithm A(p_D, p_V, x^D) (Algorithm 1, verification phase;
+ * Section 3.2).  For every position i of sequence b with mask_flags[b,i] != 0
+ * (the drafter-decoded set D of the sequence):
+ *   a_i   = argmax_x verifier_logits[b,i,x], lowest index among ties
+ *   c_i   = max_x softmax(verifier_logits[b,i,:])                    (Eq. 7)
+ *   KL_i  = KL(softmax(drafter_logits[b,i,:]) || softmax(verifier_logits[b,i,:]))
+ *           in nats                                                   (Eq. 5)
+ *   fail_i: TRUST never; KL: KL_i > tau, or u_i < KL_i / sum_{j in D} KL_j with
+ *           DD_FLAG_PROBABILISTIC (Eq. 6); CONF: c_i < tau, or u_i < 1 - c_i with
+ *           DD_FLAG_PROBABILISTIC.  u_i = (w >> 8) * 2^-24 where w is the first
+ *           word of Philox4x32-10 with key (seed low, seed high) and counter
+ *           (i, b, 0, 0).
+ *   The k positions of the sequence with the highest reliability (-KL_i or c_i,
+ *   ties to the lower i) are kept whatever fail_i says; k = 0 disables this.
+ *   out_mask[b,i]   = 1 if fail_i and not among those k, else 0
+ *   out_tokens[b,i] = tokens[b,i] if remasked (the caller overlays its [MASK]
+ *                     id) or if DD_FLAG_EMIT_DRAFTER; otherwise a_i
+ *   out_score[b,i]  = KL_i (KL mode) or c_i (CONF and TRUST modes)
+ * Positions with mask_flags == 0 pass through: out_tokens = tokens,
+ * out_mask = 0, out_score = 0, and their logits are never read.
+ *
+ * drafter_logits, verifier_logits: [B,P,V] bf16 (drafter_logits may be NULL
+ * unless the mode is KL); tokens int32 [B,P]; mask_flags uint8 [B,P];
+ * out_tokens int32 [B,P] (may alias tokens); out_mask uint8 [B,P]; out_score
+ * fp32 [B,P], nullable.  The 16-byte vector path needs V % 8 == 0 and 16-byte
+ * aligned logits; otherwise a slower element-wise path is taken.
+ * Supported: P <= 8192; V < 2^31 / 2.
+ * Errors: DD_ERR_INVALID_ARG (null required pointer, B/P/V <= 0, k < 0, unknown
+ * mode or flag bit, tau NaN), DD_ERR_UNSUPPORTED (P too large), DD_ERR_CUDA.
+ */
+int dd_verify(const void *drafter_logits, const void *verifier_logits,
+              const int32_t *tokens, const uint8_t *mask_flags,
+              int mode, float tau, int k, uint64_t seed,
+              int32_t *out_tokens, uint8_t *out_mask, float *out_score,
+              int B, int P, int V, void *stream);
+
+/*
+ * Host-buffer forms of the two calls above (same definitions, same errors).
+ * Every pointer is a HOST pointer.  The call enqueues, on `stream`, the
+ * host-to-device copies into library-owned staging memory, the kernel, and the
+ * device-to-host copies of the outputs; the outputs are valid once the stream
+ * has been synchronised by the caller.
+ */
+int dd_bidir_attention_host(const void *q, const void *k, const void *v, void *out,
+                            int B, int H, int N, int D, float scale, void *stream);
+int dd_verify_host(const void *drafter_logits, const void *verifier_logits,
+                   const int32_t *tokens, const uint8_t *mask_flags,
+                   int mode, float tau, int k, uint64_t seed,
+                   int32_t *out_tokens, uint8_t *out_mask, float *out_score,
+                   int B, int P, int V, void *stream);
+
+/* Bytes of per-device scratch dd_verify needs for this shape (informational). */
+size_t dd_verify_workspace_bytes(int B, int P, int V);
+
+/*
+ * Device-side health word of the attention kernel for the current device: 0 if
+ * no bounded wait has ever expired, otherwise a non-zero code identifying the
+ * wait that gave up (the affected output tile is then undefined).  Synchronises
+ * the device.  Returns DD_OK / DD_ERR_TIMEOUT / DD_ERR_CUDA.
+ */
+int dd_attention_status(void);
+
+/* Number of kernels launched by this library in this process (all devices). */
+uint64_t dd_launch_count(void);
+
+/* Frees the current device's scratch.  The next call re-allocates it. */
+int dd_release(void);
+
+/* Text of a dd_status; the last CUDA error text recorded by this thread. */
+const char *dd_status_string(int status);
+const char *dd_last_cuda_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int dd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DUALDIFF_H_ */

@@ -1,0 +1,156 @@
+"""CPU oracle for one DualDiffusion verification step -- TEST INFRASTRUCTURE ONLY.
+
+A ctypes loader around ``dd_oracle.c`` (plain fp64 C).  Only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import this package; the
+CUDA library never does, and this package imports nothing from it.
+
+Arrays cross the boundary as numpy arrays: bf16 tensors as ``uint16`` bit
+patterns, everything else in its natural dtype.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dd_oracle.c")
+_LIB = os.path.join(_HERE, "libdd_oracle.so")
+
+MODE_TRUST, MODE_KL, MODE_CONF = 0, 1, 2
+FLAG_PROBABILISTIC, FLAG_EMIT_DRAFTER = 0x100, 0x200
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile dd_oracle.c into libdd_oracle.so with gcc (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-Wall",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        vp, i32, f64, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_uint64
+        lib.dd_oracle_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, f64, vp, i32, vp, vp]
+        lib.dd_oracle_attention.restype = None
+        lib.dd_oracle_attention_probs.argtypes = [vp, vp, i32, i32, i32, f64, i32, i32, i32, vp]
+        lib.dd_oracle_attention_probs.restype = None
+        lib.dd_oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        lib.dd_oracle_philox4x32_10.restype = None
+        lib.dd_oracle_uniform.argtypes = [u64, i32, i32]
+        lib.dd_oracle_uniform.restype = f64
+        lib.dd_oracle_row_scores.argtypes = [vp, vp, i32, vp, vp, vp]
+        lib.dd_oracle_row_scores.restype = None
+        lib.dd_oracle_verify.argtypes = [vp, vp, vp, vp, i32, f64, i32, u64,
+                                         vp, vp, vp, vp, i32, i32, i32]
+        lib.dd_oracle_verify.restype = i32
+        lib.dd_oracle_threads.argtypes = []
+        lib.dd_oracle_threads.restype = i32
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u16(a, shape=None):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, "bf16 tensors are passed as uint16 bit patterns"
+    if shape is not None:
+        assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def threads() -> int:
+    return int(_load().dd_oracle_threads())
+
+
+def attention(q, k, v, scale, rows=None, return_lse=False):
+    """Eq. 3 over the whole key range.  q,k,v: [B,H,N,D] uint16 (bf16 bits).
+
+    Returns out [B,H,R,D] float64 (R = len(rows) or N), optionally the row LSE.
+    """
+    q = _u16(q)
+    B, H, N, D = q.shape
+    k = _u16(k, q.shape)
+    v = _u16(v, q.shape)
+    if rows is not None:
+        rows = np.ascontiguousarray(rows, dtype=np.int32)
+        assert rows.ndim == 1 and rows.size > 0 and rows.min() >= 0 and rows.max() < N
+    R = N if rows is None else rows.size
+    out = np.empty((B, H, R, D), dtype=np.float64)
+    lse = np.empty((B, H, R), dtype=np.float64)
+    _load().dd_oracle_attention(_ptr(q), _ptr(k), _ptr(v), B, H, N, D, float(scale),
+                                _ptr(rows), 0 if rows is None else rows.size,
+                                _ptr(out), _ptr(lse))
+    return (out, lse) if return_lse else out
+
+
+def attention_probs(q, k, scale, b, h, i):
+    """Softmax weights of query row i of head (b,h): float64 [N]."""
+    q = _u16(q)
+    B, H, N, D = q.shape
+    k = _u16(k, q.shape)
+    p = np.empty(N, dtype=np.float64)
+    _load().dd_oracle_attention_probs(_ptr(q), _ptr(k), H, N, D, float(scale), b, h, i, _ptr(p))
+    return p
+
+
+def philox4x32_10(counter, key):
+    c = np.ascontiguousarray(counter, dtype=np.uint32)
+    kk = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.shape == (4,) and kk.shape == (2,)
+    out = np.empty(4, dtype=np.uint32)
+    _load().dd_oracle_philox4x32_10(_ptr(c), _ptr(kk), _ptr(out))
+    return out
+
+
+def uniform(seed, b, i) -> float:
+    return float(_load().dd_oracle_uniform(int(seed), int(b), int(i)))
+
+
+def row_scores(drafter_row, verifier_row):
+    """(argmax_v, c_V, KL(p_D||p_V)) for one position; drafter_row may be None."""
+    vr = _u16(verifier_row)
+    dr = None if drafter_row is None else _u16(drafter_row, vr.shape)
+    a = ctypes.c_int32(0)
+    c = ctypes.c_double(0.0)
+    kl = ctypes.c_double(0.0)
+    _load().dd_oracle_row_scores(_ptr(dr), _ptr(vr), vr.size,
+                                 ctypes.byref(a), ctypes.byref(c), ctypes.byref(kl))
+    return int(a.value), float(c.value), float(kl.value)
+
+
+def verify(drafter, verifier, tokens, flags, mode, tau, k, seed):
+    """Verification algorithm A of Algorithm 1.  Returns a dict with
+    out_tokens int32 [B,P], out_mask uint8 [B,P], out_score float64 [B,P],
+    exempt uint8 [B,P]."""
+    verifier = _u16(verifier)
+    B, P, V = verifier.shape
+    drafter = None if drafter is None else _u16(drafter, verifier.shape)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    flags = np.ascontiguousarray(flags, dtype=np.uint8)
+    assert tokens.shape == (B, P) and flags.shape == (B, P)
+    out_tokens = np.empty((B, P), dtype=np.int32)
+    out_mask = np.empty((B, P), dtype=np.uint8)
+    out_score = np.empty((B, P), dtype=np.float64)
+    exempt = np.empty((B, P), dtype=np.uint8)
+    # tau reaches the CUDA library as a C float: the oracle compares against the same value
+    tau32 = float(np.float32(tau))
+    rc = _load().dd_oracle_verify(_ptr(drafter), _ptr(verifier), _ptr(tokens), _ptr(flags),
+                                  int(mode), tau32, int(k), int(seed),
+                                  _ptr(out_tokens), _ptr(out_mask), _ptr(out_score),
+                                  _ptr(exempt), B, P, V)
+    if rc != 0:
+        raise ValueError(f"dd_oracle_verify rejected its arguments (rc={rc})")
+    return dict(out_tokens=out_tokens, out_mask=out_mask, out_score=out_score, exempt=exempt)
