@@ -64,9 +64,9 @@ enum {
  * j over all N positions.  q, k, v, out: [B,H,N,D] bf16, D innermost, 16-byte
  * aligned, out not overlapping the inputs.  Scores and the softmax are
  * accumulated in fp32; the result is rounded to bf16 once.
- * Supported: D in {64,128}; any N >= 1; B*H*ceil(N/128) < 2^31.
+ * Supported: D in {64,128}; any N >= 1; scale >= 0; B*H*ceil(N/128) < 2^31.
  * Errors: DD_ERR_INVALID_ARG (null pointer, B/H/N/D <= 0, scale not finite),
- * DD_ERR_UNSUPPORTED (other D, misaligned pointer), DD_ERR_CUDA.
+ * DD_ERR_UNSUPPORTED (other D, negative scale, misaligned pointer), DD_ERR_CUDA.
  */
 int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
                        int B, int H, int N, int D, float scale, void *stream);

@@ -1,0 +1,169 @@
+"""Thin ctypes binding of ``include/dualdiff.h``: argument marshalling only.
+
+Every function takes torch tensors (device memory for the plain calls, pinned
+host memory for the ``*_host`` calls), passes their data pointers and sizes
+through the C ABI, and raises ``DualDiffError`` on a non-zero status.  There is
+no Python or CPU implementation behind these names: if ``libdualdiff.so`` is
+missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdualdiff.so")
+
+DD_OK, DD_ERR_INVALID_ARG, DD_ERR_UNSUPPORTED, DD_ERR_CUDA, DD_ERR_TIMEOUT = 0, -1, -2, -3, -4
+DD_MODE_TRUST, DD_MODE_KL, DD_MODE_CONF = 0, 1, 2
+DD_FLAG_PROBABILISTIC, DD_FLAG_EMIT_DRAFTER = 0x100, 0x200
+
+# every symbol include/dualdiff.h declares
+EXPORTS = (
+    "dd_bidir_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host",
+    "dd_verify_workspace_bytes", "dd_attention_status", "dd_launch_count", "dd_release",
+    "dd_status_string", "dd_last_cuda_error", "dd_version",
+)
+
+
+class DualDiffError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"dualdiff status {status}: {text}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdualdiff.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2604_05250_b200.build`; "
+                "there is no fallback implementation")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, f32, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint64
+        attn = [vp, vp, vp, vp, i32, i32, i32, i32, f32, vp]
+        ver = [vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, vp]
+        L.dd_bidir_attention.argtypes = attn
+        L.dd_bidir_attention_host.argtypes = attn
+        L.dd_verify.argtypes = ver
+        L.dd_verify_host.argtypes = ver
+        for name in ("dd_bidir_attention", "dd_bidir_attention_host", "dd_verify", "dd_verify_host",
+                     "dd_attention_status", "dd_release", "dd_version"):
+            getattr(L, name).restype = i32
+        L.dd_attention_status.argtypes = []
+        L.dd_release.argtypes = []
+        L.dd_version.argtypes = []
+        L.dd_verify_workspace_bytes.argtypes = [i32, i32, i32]
+        L.dd_verify_workspace_bytes.restype = ctypes.c_size_t
+        L.dd_launch_count.argtypes = []
+        L.dd_launch_count.restype = u64
+        L.dd_status_string.argtypes = [i32]
+        L.dd_status_string.restype = ctypes.c_char_p
+        L.dd_last_cuda_error.argtypes = []
+        L.dd_last_cuda_error.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(status: int):
+    if status != DD_OK:
+        L = lib()
+        text = L.dd_status_string(status).decode()
+        if status == DD_ERR_CUDA:
+            text += ": " + L.dd_last_cuda_error().decode()
+        raise DualDiffError(status, text)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _require(t, dtype, shape, cuda, name):
+    import torch
+    if not isinstance(t, torch.Tensor):
+        raise TypeError(f"{name}: expected a torch.Tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError(f"{name}: expected contiguous {dtype} of shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)}")
+    if t.is_cuda != cuda:
+        raise ValueError(f"{name}: expected a {'device' if cuda else 'host'} tensor")
+
+
+def bidir_attention(q, k, v, out=None, scale=None, stream=None, host=False):
+    """dd_bidir_attention (dd_bidir_attention_host if host=True).
+
+    q, k, v: [B,H,N,D] torch.bfloat16.  Returns out (allocated if None)."""
+    import torch
+    B, H, N, D = q.shape
+    cuda = not host
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _require(t, torch.bfloat16, (B, H, N, D), cuda, name)
+    if out is None:
+        out = torch.empty_like(q)
+    _require(out, torch.bfloat16, (B, H, N, D), cuda, "out")
+    if scale is None:
+        scale = float(D) ** -0.5
+    fn = lib().dd_bidir_attention_host if host else lib().dd_bidir_attention
+    _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale), _stream_ptr(stream)))
+    return out
+
+
+def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, seed,
+           out_tokens=None, out_mask=None, out_score=None, want_score=True, stream=None, host=False):
+    """dd_verify (dd_verify_host if host=True).
+
+    Returns (out_tokens int32 [B,P], out_mask uint8 [B,P], out_score float32 [B,P] or None)."""
+    import torch
+    B, P, V = verifier_logits.shape
+    cuda = not host
+    _require(verifier_logits, torch.bfloat16, (B, P, V), cuda, "verifier_logits")
+    if drafter_logits is not None:
+        _require(drafter_logits, torch.bfloat16, (B, P, V), cuda, "drafter_logits")
+    _require(tokens, torch.int32, (B, P), cuda, "tokens")
+    _require(mask_flags, torch.uint8, (B, P), cuda, "mask_flags")
+    kw = dict(device=verifier_logits.device, pin_memory=host)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, P), dtype=torch.int32, **kw)
+    if out_mask is None:
+        out_mask = torch.empty((B, P), dtype=torch.uint8, **kw)
+    if out_score is None and want_score:
+        out_score = torch.empty((B, P), dtype=torch.float32, **kw)
+    _require(out_tokens, torch.int32, (B, P), cuda, "out_tokens")
+    _require(out_mask, torch.uint8, (B, P), cuda, "out_mask")
+    if out_score is not None:
+        _require(out_score, torch.float32, (B, P), cuda, "out_score")
+    fn = lib().dd_verify_host if host else lib().dd_verify
+    _check(fn(_ptr(drafter_logits), _ptr(verifier_logits), _ptr(tokens), _ptr(mask_flags),
+              int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
+              _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, V, _stream_ptr(stream)))
+    return out_tokens, out_mask, out_score
+
+
+def attention_status() -> int:
+    return int(lib().dd_attention_status())
+
+
+def launch_count() -> int:
+    return int(lib().dd_launch_count())
+
+
+def release():
+    _check(lib().dd_release())
+
+
+def version() -> int:
+    return int(lib().dd_version())
+
+
+def verify_workspace_bytes(B, P, V) -> int:
+    return int(lib().dd_verify_workspace_bytes(B, P, V))

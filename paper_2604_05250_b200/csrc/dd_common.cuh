@@ -1,0 +1,40 @@
+// Shared host-side plumbing of the library: status codes, per-device scratch,
+// CUDA error capture, launch counting.  No kernel arithmetic lives here.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/dualdiff.h"
+
+namespace dd {
+
+// Per-device scratch owned by the library.
+struct DeviceCtx {
+    void *verify_ws = nullptr;      // dd_verify partials, counters, row results
+    size_t verify_ws_bytes = 0;
+    void *staging = nullptr;        // device copies of host buffers (the *_host calls)
+    size_t staging_bytes = 0;
+    unsigned int *attn_status = nullptr;  // one word: first expired wait of the attention kernel
+};
+
+// Returns the context of the current device (creating it on first use), or
+// nullptr after recording a CUDA error.
+DeviceCtx *current_ctx(int *device_out = nullptr);
+
+// Grows (never shrinks) a scratch buffer; new memory is zero-filled.
+int ensure_bytes(void **ptr, size_t *have, size_t need);
+
+// Records a CUDA error text for dd_last_cuda_error() and returns DD_ERR_CUDA.
+int cuda_fail(cudaError_t e, const char *where);
+
+void count_launch(unsigned n = 1);
+
+#define DD_CUDA_TRY(expr)                                         \
+    do {                                                          \
+        cudaError_t _e = (expr);                                  \
+        if (_e != cudaSuccess) return ::dd::cuda_fail(_e, #expr); \
+    } while (0)
+
+}  // namespace dd

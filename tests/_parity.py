@@ -1,0 +1,61 @@
+"""Shared comparison rules of the GPU parity tests.
+
+Attention: max-abs <= 1e-2 and mean-abs <= 1e-3 against the fp64 oracle.
+Verify: scores within 1e-4 relative (absolute floor 1e-6 where the score is
+near zero); remask sets and emitted tokens bit-exact except at positions the
+oracle flags as lying within 1e-5 of a decision boundary.
+"""
+import numpy as np
+
+ATTN_MAX_ABS = 1e-2
+ATTN_MEAN_ABS = 1e-3
+SCORE_REL = 1e-4
+SCORE_ABS_FLOOR = 1e-6
+
+
+def to_torch_bf16(bits, device=None, pin=False):
+    import torch
+    t = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    if device is not None:
+        return t.to(device)
+    return t.pin_memory() if pin else t
+
+
+def bf16_tensor_to_f64(t):
+    import torch
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def check_attention(gpu_out_f64, oracle_out):
+    diff = np.abs(gpu_out_f64 - oracle_out)
+    assert np.isfinite(gpu_out_f64).all()
+    assert diff.max() <= ATTN_MAX_ABS, f"max-abs {diff.max():.3e}"
+    assert diff.mean() <= ATTN_MEAN_ABS, f"mean-abs {diff.mean():.3e}"
+    return float(diff.max()), float(diff.mean())
+
+
+def check_verify(gpu_tokens, gpu_mask, gpu_score, ref, flags, tokens_in):
+    """ref: dict from oracle.verify; gpu_*: numpy arrays."""
+    flags = flags.astype(bool)
+    exempt = ref["exempt"].astype(bool)
+    o_score = ref["out_score"]
+    tol = np.maximum(SCORE_REL * np.abs(o_score), SCORE_ABS_FLOOR)
+    bad = np.abs(gpu_score.astype(np.float64) - o_score) > tol
+    assert not bad.any(), (f"{bad.sum()} scores out of tolerance; worst "
+                           f"{np.abs(gpu_score - o_score).max():.3e}")
+    strict = ~exempt
+    mism_mask = (gpu_mask != ref["out_mask"]) & strict
+    assert not mism_mask.any(), f"{mism_mask.sum()} remask decisions differ outside the exempt set"
+    mism_tok = (gpu_tokens != ref["out_tokens"]) & strict
+    assert not mism_tok.any(), f"{mism_tok.sum()} emitted tokens differ outside the exempt set"
+    # at exempt positions either decision is acceptable, but the token must match that decision
+    ex = exempt & flags
+    if ex.any():
+        kept_tok = np.where(ref["out_mask"].astype(bool), -1, ref["out_tokens"])
+        ok = (gpu_mask.astype(bool) & (gpu_tokens == tokens_in)) | \
+             (~gpu_mask.astype(bool) & ((gpu_tokens == kept_tok) | (kept_tok < 0)))
+        assert ok[ex].all()
+    # unflagged positions pass through untouched
+    assert (gpu_tokens[~flags] == tokens_in[~flags]).all()
+    assert not gpu_mask[~flags].any() and not gpu_score[~flags].any()
+    return int(exempt.sum())

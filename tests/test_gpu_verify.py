@@ -1,0 +1,192 @@
+"""dd_verify on the GPU against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2604_05250_b200 import synth
+from tests._parity import check_verify, to_torch_bf16
+
+pytestmark = pytest.mark.gpu
+
+TRUST, KL, CONF = 0, 1, 2
+PROB, EMIT = 0x100, 0x200
+
+
+@pytest.fixture(scope="module")
+def dd():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2604_05250_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def run_gpu(dd, dra, ver, tokens, flags, mode, tau, k, seed, host=False):
+    import torch
+    dev = None if host else "cuda"
+    t_ver = to_torch_bf16(ver, dev, pin=host)
+    t_dra = None if dra is None else to_torch_bf16(dra, dev, pin=host)
+    t_tok = torch.from_numpy(tokens)
+    t_fl = torch.from_numpy(flags)
+    if host:
+        t_tok, t_fl = t_tok.pin_memory(), t_fl.pin_memory()
+    else:
+        t_tok, t_fl = t_tok.cuda(), t_fl.cuda()
+    ot, om, osc = dd.verify(t_dra, t_ver, t_tok, t_fl, mode, tau, k, seed, host=host)
+    torch.cuda.synchronize()
+    return ot.cpu().numpy(), om.cpu().numpy(), osc.cpu().numpy()
+
+
+def compare(dd, oracle_mod, dra, ver, tokens, flags, mode, tau, k, seed, host=False):
+    algo = mode & 0xFF
+    d_in = dra if algo == KL else None
+    ref = oracle_mod.verify(d_in, ver, tokens, flags, mode, tau, k, seed)
+    ot, om, osc = run_gpu(dd, d_in, ver, tokens, flags, mode, tau, k, seed, host=host)
+    return check_verify(ot, om, osc, ref, flags, tokens), ref, (ot, om, osc)
+
+
+ALL_MODES = [TRUST, KL, CONF, KL | PROB, CONF | PROB, KL | EMIT, TRUST | EMIT, CONF | PROB | EMIT]
+
+
+@pytest.mark.parametrize("mode", ALL_MODES)
+def test_config0_tiny(dd, oracle_mod, mode):
+    c = synth.VERIFY_CONFIGS[0]
+    dra, ver, tokens, flags = synth.verify_config_inputs(0)
+    assert flags.sum() == 32
+    compare(dd, oracle_mod, dra, ver, tokens, flags, mode, c["tau"], c["k"], c["seed"])
+
+
+@pytest.mark.parametrize("V", [8, 1000, 1003, 8192, 8200, 8201, 20000, 32000])
+@pytest.mark.parametrize("mode", [KL, CONF])
+def test_vocab_sizes_and_ragged_tails(dd, oracle_mod, V, mode):
+    """Several chunks plus a ragged tail; V % 8 != 0 takes the element-wise path."""
+    dra, ver, tokens, flags = synth.verify_inputs(2, 24, V, 17, 0.2, seed=V)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, mode, 0.5, 4, 1)
+
+
+def test_config1_llada_shaped_full_size(dd, oracle_mod):
+    c = synth.VERIFY_CONFIGS[1]
+    dra, ver, tokens, flags = synth.verify_config_inputs(1)
+    n_ex, ref, _ = compare(dd, oracle_mod, dra, ver, tokens, flags, KL, c["tau"], c["k"], c["seed"])
+    assert 5 <= ref["out_mask"].sum() <= 60           # ~10% drafter errors get remasked
+    assert n_ex <= 4
+    # probabilistic variant and the host-buffer entry point on the same data
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL | PROB, c["tau"], c["k"], 3)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL, c["tau"], c["k"], c["seed"], host=True)
+
+
+def test_config2_batched_full_size(dd, oracle_mod):
+    c = synth.VERIFY_CONFIGS[2]
+    dra, ver, tokens, flags = synth.verify_config_inputs(2)
+    counts = flags.sum(axis=1)
+    assert counts.min() >= 64 and counts.max() <= 256 and len(set(counts.tolist())) > 4
+    _, ref, _ = compare(dd, oracle_mod, dra, ver, tokens, flags, CONF, c["tau"], c["k"], c["seed"])
+    # every position fails c < 0.5 at this vocabulary size: the top-k rule decides
+    kept = (flags.astype(bool) & ~ref["out_mask"].astype(bool)).sum(axis=1)
+    assert (kept == c["k"]).all()
+    compare(dd, oracle_mod, dra, ver, tokens, flags, CONF | PROB, c["tau"], c["k"], 5)
+
+
+@pytest.mark.parametrize("mode", [TRUST, KL])
+def test_config3_long_context(dd, oracle_mod, mode):
+    c = synth.VERIFY_CONFIGS[3]
+    dra, ver, tokens, flags = synth.verify_config_inputs(3)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, mode, c["tau"], c["k"], c["seed"])
+
+
+@pytest.mark.parametrize("V,seeds", [(32000, (0, 1, 2, 3)), (126464, (0,))])
+@pytest.mark.parametrize("err", [0.05, 0.20, 0.50])
+def test_config4_sweep(dd, oracle_mod, V, seeds, err):
+    sw = synth.VERIFY_SWEEP
+    for seed in seeds:
+        for nflag in sw["flagged"]:
+            dra, ver, tokens, flags = synth.verify_inputs(1, sw["P"], V, nflag, err,
+                                                          synth.config_seed(4, seed))
+            k = 8 if nflag == 32 else 32
+            for mode in (TRUST, KL, CONF) if seed == 0 else (KL,):
+                compare(dd, oracle_mod, dra, ver, tokens, flags, mode, sw["tau"], k, seed)
+            if seed == 0 and nflag == 128:
+                compare(dd, oracle_mod, dra, ver, tokens, flags, KL | PROB, sw["tau"], k, seed)
+                compare(dd, oracle_mod, dra, ver, tokens, flags, CONF | PROB, sw["tau"], k, seed)
+
+
+def test_degenerate_cases(dd, oracle_mod):
+    dra, ver, tokens, flags = synth.verify_inputs(3, 16, 256, 9, 0.3, seed=11)
+    # nothing flagged anywhere: pure pass-through
+    none = np.zeros_like(flags)
+    compare(dd, oracle_mod, dra, ver, tokens, none, KL, 0.5, 4, 0)
+    # one sequence empty, one full
+    mixed = flags.copy(); mixed[0] = 0; mixed[1] = 1
+    compare(dd, oracle_mod, dra, ver, tokens, mixed, KL, 0.5, 4, 0)
+    # k = 0 (pure rule), k >= number flagged (keep all), unreachable thresholds
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.05, 0, 0)
+    _, ref, got = compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.0, 1000, 0)
+    assert not got[1].any()
+    compare(dd, oracle_mod, dra, ver, tokens, flags, CONF, 2.0, 3, 0)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 1e9, 3, 0)
+    # identical drafter and verifier: KL = 0 everywhere, nothing exceeds tau = 0
+    _, ref, got = compare(dd, oracle_mod, ver, ver, tokens, flags, KL, 0.0, 0, 0)
+    assert not got[1].any() and np.abs(got[2]).max() <= 1e-6
+    # P = 1, V = 8
+    d1, v1, t1, f1 = synth.verify_inputs(1, 1, 8, 1, 0.0, seed=12)
+    compare(dd, oracle_mod, d1, v1, t1, f1, CONF, 0.5, 0, 0)
+
+
+def test_exact_ties_in_verifier_row(dd, oracle_mod):
+    dra, ver, tokens, flags = synth.verify_inputs(1, 8, 20000, 8, 0.0, seed=13)
+    top = synth.f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    ver[0, 0, [19999, 8191, 8192, 12345]] = top        # ties across chunk and warp boundaries
+    ver[0, 1, [7, 3]] = top
+    ver[0, 2, :] = top                                  # a constant row
+    _, ref, got = compare(dd, oracle_mod, dra, ver, tokens, flags, TRUST, 0.5, 0, 0)
+    assert got[0][0, 0] == 8191 and got[0][0, 1] == 3 and got[0][0, 2] == 0
+
+
+def test_threshold_sweep_crosses_scores(dd, oracle_mod):
+    """Thresholds placed on and next to actual scores exercise the exempt band."""
+    dra, ver, tokens, flags = synth.verify_inputs(1, 32, 4096, 32, 0.3, seed=14)
+    ref = oracle_mod.verify(dra, ver, tokens, flags, KL, 0.5, 0, 0)
+    scores = np.sort(ref["out_score"][0])
+    n_exempt = 0
+    for s in scores[::4]:
+        for tau in (s, s * (1 + 3e-6), s * (1 - 3e-6), s + 1e-3):
+            n, _, _ = compare(dd, oracle_mod, dra, ver, tokens, flags, KL, float(tau), 0, 0)
+            n_exempt += n
+    assert n_exempt > 0
+
+
+def test_out_tokens_may_alias_tokens_and_score_is_optional(dd, oracle_mod):
+    import torch
+    dra, ver, tokens, flags = synth.verify_inputs(2, 16, 1024, 10, 0.2, seed=15)
+    ref = oracle_mod.verify(dra, ver, tokens, flags, KL, 0.5, 2, 0)
+    t_tok = torch.from_numpy(tokens.copy()).cuda()
+    ot, om, osc = dd.verify(to_torch_bf16(dra, "cuda"), to_torch_bf16(ver, "cuda"), t_tok,
+                            torch.from_numpy(flags).cuda(), KL, 0.5, 2, 0,
+                            out_tokens=t_tok, want_score=False)
+    torch.cuda.synchronize()
+    assert osc is None
+    strict = ~ref["exempt"].astype(bool)
+    assert (ot.cpu().numpy()[strict] == ref["out_tokens"][strict]).all()
+    assert (om.cpu().numpy()[strict] == ref["out_mask"][strict]).all()
+
+
+def test_bitwise_repeatability(dd, oracle_mod):
+    dra, ver, tokens, flags = synth.verify_inputs(4, 64, 32000, "uniform_25_100", 0.2, seed=16)
+    first = run_gpu(dd, dra, ver, tokens, flags, KL | PROB, 0.5, 8, 9)
+    for _ in range(5):
+        again = run_gpu(dd, dra, ver, tokens, flags, KL | PROB, 0.5, 8, 9)
+        for a, b in zip(first, again):
+            assert np.array_equal(a, b)
+
+
+def test_philox_stream_matches_oracle(dd, oracle_mod):
+    """With all verifier logits equal, c = 1/2 exactly at V = 2... use V = 8: c = 1/8, so
+    CONF|PROB remasks iff u < 7/8: the GPU's uniforms must match the oracle's one by one."""
+    B, P, V = 3, 200, 8
+    ver = np.zeros((B, P, V), dtype=np.uint16)
+    tokens = np.zeros((B, P), dtype=np.int32)
+    flags = np.ones((B, P), dtype=np.uint8)
+    for seed in (0, 1, 0xDEADBEEFCAFEF00D):
+        ot, om, osc = run_gpu(dd, None, ver, tokens, flags, CONF | PROB, 0.5, 0, seed)
+        expect = np.array([[oracle_mod.uniform(seed, b, i) < 0.875 for i in range(P)] for b in range(B)])
+        assert np.array_equal(om.astype(bool), expect)
