@@ -91,6 +91,7 @@ int dd_release(void)
     if (!ctx) return DD_ERR_CUDA;
     DD_CUDA_TRY(cudaDeviceSynchronize());
     if (ctx->verify_ws) DD_CUDA_TRY(cudaFree(ctx->verify_ws));
+    if (ctx->verify_cnt) DD_CUDA_TRY(cudaFree(ctx->verify_cnt));
     if (ctx->staging) DD_CUDA_TRY(cudaFree(ctx->staging));
     if (ctx->attn_status) DD_CUDA_TRY(cudaFree(ctx->attn_status));
     *ctx = DeviceCtx();

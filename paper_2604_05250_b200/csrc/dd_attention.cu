@@ -142,8 +142,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         float mx = -INFINITY;
 #pragma unroll
         for (int i = 0; i < kBlockN; ++i) {
-            if (i >= valid) s[i] = -INFINITY;
-            mx = fmaxf(mx, s[i]);
+            if (i < valid) mx = fmaxf(mx, s[i]);
         }
         const float m_new = fmaxf(m_run, mx * p.scale_log2);
         const float alpha = ex2(m_run - m_new);
@@ -151,8 +150,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         uint32_t pk[kBlockN / 2];
 #pragma unroll
         for (int i = 0; i < kBlockN; i += 2) {
-            const float p0 = ex2(fmaf(s[i], p.scale_log2, -m_new));
-            const float p1 = ex2(fmaf(s[i + 1], p.scale_log2, -m_new));
+            // keys past the end of the sequence get weight zero (no -inf arithmetic: scale may be 0)
+            const float p0 = i < valid ? ex2(fmaf(s[i], p.scale_log2, -m_new)) : 0.f;
+            const float p1 = i + 1 < valid ? ex2(fmaf(s[i + 1], p.scale_log2, -m_new)) : 0.f;
             sum += p0 + p1;
             __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
             pk[i / 2] = *reinterpret_cast<uint32_t *>(&h);

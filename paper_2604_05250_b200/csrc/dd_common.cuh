@@ -12,8 +12,10 @@ namespace dd {
 
 // Per-device scratch owned by the library.
 struct DeviceCtx {
-    void *verify_ws = nullptr;      // dd_verify partials, counters, row results
+    void *verify_ws = nullptr;      // dd_verify chunk partials and row results
     size_t verify_ws_bytes = 0;
+    void *verify_cnt = nullptr;     // dd_verify completion counters: all zero between launches
+    size_t verify_cnt_bytes = 0;
     void *staging = nullptr;        // device copies of host buffers (the *_host calls)
     size_t staging_bytes = 0;
     unsigned int *attn_status = nullptr;  // one word: first expired wait of the attention kernel

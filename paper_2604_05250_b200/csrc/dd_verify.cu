@@ -431,12 +431,18 @@ __global__ void __launch_bounds__(kThreads, KL ? 3 : 4) verify_kernel(const Veri
     decide_sequence(p, b, keys, red);
 }
 
+// Counters live in their own allocation: it holds nothing else, so it is all zero whenever no
+// launch is in flight, whatever (B, P) the previous call used.
+size_t counter_bytes(int B, int P)
+{
+    const size_t bp = (size_t)B * P;
+    return ((bp * 4 + 255) & ~size_t(255)) + (((size_t)B * 4 + 255) & ~size_t(255));
+}
+
 size_t workspace_bytes(int B, int P, int nchunks)
 {
     const size_t bp = (size_t)B * P;
     size_t bytes = 0;
-    bytes += (bp * 4 + 255) & ~size_t(255);           // row_counter
-    bytes += ((size_t)B * 4 + 255) & ~size_t(255);    // seq_counter
     bytes += (bp * 4 + 255) & ~size_t(255);           // row_score
     bytes += (bp * 4 + 255) & ~size_t(255);           // row_argmax
     bytes += bp * nchunks * sizeof(Partial);
@@ -477,7 +483,7 @@ extern "C" size_t dd_verify_workspace_bytes(int B, int P, int V)
     if (B <= 0 || P <= 0 || V <= 0) return 0;
     int nchunks, chunk;
     chunking(V, &nchunks, &chunk);
-    return workspace_bytes(B, P, nchunks);
+    return workspace_bytes(B, P, nchunks) + counter_bytes(B, P);
 }
 
 extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits,
@@ -504,11 +510,13 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     if (!ctx) return DD_ERR_CUDA;
     int rc = dd::ensure_bytes(&ctx->verify_ws, &ctx->verify_ws_bytes, workspace_bytes(B, P, p.nchunks));
     if (rc != DD_OK) return rc;
+    rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(B, P));
+    if (rc != DD_OK) return rc;
 
     const size_t bp = (size_t)B * P;
+    p.row_counter = (unsigned int *)ctx->verify_cnt;
+    p.seq_counter = (unsigned int *)((char *)ctx->verify_cnt + ((bp * 4 + 255) & ~size_t(255)));
     char *w = (char *)ctx->verify_ws;
-    p.row_counter = (unsigned int *)w; w += (bp * 4 + 255) & ~size_t(255);
-    p.seq_counter = (unsigned int *)w; w += ((size_t)B * 4 + 255) & ~size_t(255);
     p.row_score = (float *)w;          w += (bp * 4 + 255) & ~size_t(255);
     p.row_argmax = (int *)w;           w += (bp * 4 + 255) & ~size_t(255);
     p.partials = (Partial *)w;

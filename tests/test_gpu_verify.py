@@ -190,3 +190,12 @@ def test_philox_stream_matches_oracle(dd, oracle_mod):
         ot, om, osc = run_gpu(dd, None, ver, tokens, flags, CONF | PROB, 0.5, 0, seed)
         expect = np.array([[oracle_mod.uniform(seed, b, i) < 0.875 for i in range(P)] for b in range(B)])
         assert np.array_equal(om.astype(bool), expect)
+
+
+def test_scratch_survives_changing_shapes(dd, oracle_mod):
+    """Calls of different (B, P, V) in a row reuse the library's scratch: the completion
+    counters must not inherit stale data from a previous layout."""
+    shapes = [(1, 8, 64), (4, 300, 1024), (2, 16, 20000), (6, 700, 256), (1, 8, 64), (3, 200, 8)]
+    for n, (B, P, V) in enumerate(shapes):
+        dra, ver, tokens, flags = synth.verify_inputs(B, P, V, max(1, P // 2), 0.2, seed=100 + n)
+        compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 3, n)
