@@ -123,6 +123,30 @@ int dd_verify_host(const void *drafter_logits, const void *verifier_logits,
                    int32_t *out_tokens, uint8_t *out_mask, float *out_score,
                    int B, int P, int V, void *stream);
 
+/*
+ * dd_verify for callers that must not allocate device memory (the paper has no
+ * counterpart to this entry point; it is the same computation as dd_verify, with
+ * the same arguments, outputs and errors).  Meant for code that runs inside a
+ * fixed memory budget, that may not trigger the device-wide synchronisation of
+ * cudaMalloc/cudaFree, or that does not own the allocator of its process: this
+ * call performs no cudaMalloc, cudaFree or other allocating routine.  Its scratch
+ * (chunk partials, row results, completion counters) is a fixed array of about
+ * 2.1 MB inside the library, held by every GPU that loads the library until the
+ * process exits.
+ * Limits: B*P <= 4096 and B*P*ceil(V/8192) <= 65536; larger problems return
+ * DD_ERR_UNSUPPORTED and launch nothing.
+ * The first call on each device looks up the array's device address; make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array: each call clears the counters it needs on `stream` before its kernel,
+ * and two calls that may overlap on the GPU (different streams without ordering)
+ * race on the scratch and give undefined results.
+ */
+int dd_verify_static(const void *drafter_logits, const void *verifier_logits,
+                     const int32_t *tokens, const uint8_t *mask_flags,
+                     int mode, float tau, int k, uint64_t seed,
+                     int32_t *out_tokens, uint8_t *out_mask, float *out_score,
+                     int B, int P, int V, void *stream);
+
 /* Bytes of per-device scratch dd_verify needs for this shape (informational). */
 size_t dd_verify_workspace_bytes(int B, int P, int V);
 

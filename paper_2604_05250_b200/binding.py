@@ -20,7 +20,7 @@ DD_FLAG_PROBABILISTIC, DD_FLAG_EMIT_DRAFTER = 0x100, 0x200
 
 # every symbol include/dualdiff.h declares
 EXPORTS = (
-    "dd_bidir_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host",
+    "dd_bidir_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_launch_count", "dd_release",
     "dd_status_string", "dd_last_cuda_error", "dd_version",
 )
@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.dd_bidir_attention_host.argtypes = attn
         L.dd_verify.argtypes = ver
         L.dd_verify_host.argtypes = ver
+        L.dd_verify_static.argtypes = ver
+        L.dd_verify_static.restype = i32
         for name in ("dd_bidir_attention", "dd_bidir_attention_host", "dd_verify", "dd_verify_host",
                      "dd_attention_status", "dd_release", "dd_version"):
             getattr(L, name).restype = i32
@@ -119,8 +121,10 @@ def bidir_attention(q, k, v, out=None, scale=None, stream=None, host=False):
 
 
 def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, seed,
-           out_tokens=None, out_mask=None, out_score=None, want_score=True, stream=None, host=False):
-    """dd_verify (dd_verify_host if host=True).
+           out_tokens=None, out_mask=None, out_score=None, want_score=True, stream=None, host=False,
+           static_scratch=False):
+    """dd_verify (dd_verify_host if host=True; dd_verify_static, the variant that allocates
+    nothing, if static_scratch=True and every output tensor is passed in).
 
     Returns (out_tokens int32 [B,P], out_mask uint8 [B,P], out_score float32 [B,P] or None)."""
     import torch
@@ -142,7 +146,7 @@ def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, se
     _require(out_mask, torch.uint8, (B, P), cuda, "out_mask")
     if out_score is not None:
         _require(out_score, torch.float32, (B, P), cuda, "out_score")
-    fn = lib().dd_verify_host if host else lib().dd_verify
+    fn = lib().dd_verify_host if host else (lib().dd_verify_static if static_scratch else lib().dd_verify)
     _check(fn(_ptr(drafter_logits), _ptr(verifier_logits), _ptr(tokens), _ptr(mask_flags),
               int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
               _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, V, _stream_ptr(stream)))

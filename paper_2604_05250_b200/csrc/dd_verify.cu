@@ -545,3 +545,99 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     if (kl) return vec ? launch<true, true>(p, smem, s) : launch<true, false>(p, smem, s);
     return vec ? launch<false, true>(p, smem, s) : launch<false, false>(p, smem, s);
 }
+
+// ---------------------------------------------------------------------------
+// dd_verify_static: the same kernel with its scratch in a fixed device array.
+//
+// Some callers must not allocate device memory at all: code running inside a
+// pre-sized memory budget (an inference server that has handed every free byte
+// to its KV cache), code that may not trigger the implicit device
+// synchronisation of cudaMalloc/cudaFree, or a process whose allocator is owned
+// by another runtime.  For them the partials, row results and completion
+// counters live in the file-scope array below, which every GPU that loads this
+// library holds until the process exits.
+namespace {
+
+constexpr int kStaticMaxRows = 4096;          // B * P
+constexpr int kStaticMaxPartials = 65536;     // B * P * ceil(V / 8192)
+constexpr size_t kStaticCounterBytes = (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255)) +
+                                       (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));   // rows + sequences
+constexpr size_t kStaticRowBytes = 2 * (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));  // score + argmax
+constexpr size_t kStaticScratchBytes = kStaticCounterBytes + kStaticRowBytes +
+                                       (size_t)kStaticMaxPartials * sizeof(Partial);
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address to pass on.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch per device, resolved on the first call made on that device.
+unsigned char *g_static_ptr[64] = {};
+
+}  // namespace
+
+extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier_logits,
+                                const int32_t *tokens, const uint8_t *mask_flags,
+                                int mode, float tau, int k, uint64_t seed,
+                                int32_t *out_tokens, uint8_t *out_mask, float *out_score,
+                                int B, int P, int V, void *stream)
+{
+    const int algo = mode & 0xFF;
+    if (!verifier_logits || !tokens || !mask_flags || !out_tokens || !out_mask) return DD_ERR_INVALID_ARG;
+    if (B <= 0 || P <= 0 || V <= 0 || k < 0) return DD_ERR_INVALID_ARG;
+    if (algo != DD_MODE_TRUST && algo != DD_MODE_KL && algo != DD_MODE_CONF) return DD_ERR_INVALID_ARG;
+    if (mode & ~(0xFF | DD_FLAG_PROBABILISTIC | DD_FLAG_EMIT_DRAFTER)) return DD_ERR_INVALID_ARG;
+    if (algo == DD_MODE_KL && !drafter_logits) return DD_ERR_INVALID_ARG;
+    if (tau != tau) return DD_ERR_INVALID_ARG;
+    if (P > kMaxP) return DD_ERR_UNSUPPORTED;
+    if ((long)V >= (1L << 30)) return DD_ERR_UNSUPPORTED;
+
+    VerifyParams p;
+    chunking(V, &p.nchunks, &p.chunk);
+    // the fixed scratch bounds the problem size
+    if ((long)B * P > kStaticMaxRows || (long)B * P * p.nchunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
+
+    int dev = -1;
+    DD_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return dd::cuda_fail(cudaErrorInvalidDevice, "dd_verify_static: device index");
+    if (!g_static_ptr[dev]) {
+        // set-up, once per device, with that device current
+        void *ptr = nullptr;
+        DD_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_ptr[dev] = static_cast<unsigned char *>(ptr);
+    }
+    unsigned char *base = g_static_ptr[dev];
+    const size_t bp = (size_t)B * P;
+    const size_t rows_slot = ((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255);
+    p.row_counter = (unsigned int *)base;
+    p.seq_counter = (unsigned int *)(base + rows_slot);
+    p.row_score = (float *)(base + kStaticCounterBytes);
+    p.row_argmax = (int *)(base + kStaticCounterBytes + rows_slot);
+    p.partials = (Partial *)(base + kStaticCounterBytes + kStaticRowBytes);
+
+    p.drafter = (const uint16_t *)drafter_logits;
+    p.verifier = (const uint16_t *)verifier_logits;
+    p.tokens = tokens;
+    p.flags = mask_flags;
+    p.out_tokens = out_tokens;
+    p.out_mask = out_mask;
+    p.out_score = out_score;
+    p.B = B; p.P = P; p.V = V;
+    p.algo = algo;
+    p.probabilistic = (mode & DD_FLAG_PROBABILISTIC) != 0;
+    p.emit_drafter = (mode & DD_FLAG_EMIT_DRAFTER) != 0;
+    p.tau = tau;
+    p.k = k;
+    p.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu);
+    p.seed_hi = (uint32_t)(seed >> 32);
+
+    cudaStream_t s = (cudaStream_t)stream;
+    // The array keeps whatever the previous call left: the counters must start at zero.
+    DD_CUDA_TRY(cudaMemsetAsync(p.row_counter, 0, bp * 4, s));
+    DD_CUDA_TRY(cudaMemsetAsync(p.seq_counter, 0, (size_t)B * 4, s));
+
+    const bool kl = algo == DD_MODE_KL;
+    const bool vec = (V % 8 == 0) && (((uintptr_t)verifier_logits & 15) == 0) &&
+                     (!kl || ((uintptr_t)drafter_logits & 15) == 0);
+    const size_t smem = (size_t)P * sizeof(unsigned long long);
+    if (kl) return vec ? launch<true, true>(p, smem, s) : launch<true, false>(p, smem, s);
+    return vec ? launch<false, true>(p, smem, s) : launch<false, false>(p, smem, s);
+}
