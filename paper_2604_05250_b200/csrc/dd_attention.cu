@@ -1,16 +1,22 @@
 // dd_bidir_attention: full-sequence bidirectional attention (Section 2.2; Eq. 3
 // evaluated over the whole key range) for sm_100a.
 //
-// One CTA owns a tile of 128 query rows of one (batch, head) and walks over the
-// keys in tiles of 128.  Q, K and V tiles arrive in shared memory by TMA (3-D
-// tensor maps over [B*H, N, D], 128-byte swizzle; rows past N read as zero).
-// S = Q K^T is a tcgen05 MMA into tensor memory; each of the 128 threads owns one
-// query row (= one TMEM lane), reads its 128 scores, keeps the running row
-// maximum and sum in fp32 (online softmax, base 2 with scale*log2e folded in),
-// writes P = 2^(S - m) as bf16 back into the same TMEM columns, and O += P V is a
-// second tcgen05 MMA whose A operand is read from TMEM.  O is rescaled in TMEM
-// when the row maximum moves, normalised by the row sum at the end and rounded to
-// bf16 once.
+// One CTA owns two tiles of 128 query rows of one (batch, head) and walks over
+// the keys in tiles of 128.  The CTA is warp-specialised:
+//   warps 0-3   softmax of query tile 0 (thread = query row = TMEM lane)
+//   warps 4-7   softmax of query tile 1
+//   warp  8     one thread feeds a ring of K/V tiles by TMA (3-D tensor maps over
+//               [B*H, N, D], 128-byte swizzle; rows past N read as zero)
+//   warp  9     one thread issues every tcgen05 MMA
+// S_g = Q_g K^T goes to tensor memory; the softmax thread reads its row, keeps the
+// running maximum and sum in fp32 (online softmax in base 2, scale*log2e folded
+// into one FMA), writes P = 2^(S - m) as bf16 over the first half of the S columns,
+// and O_g += P V is a second MMA whose A operand is read from tensor memory.  While
+// one tile's softmax runs, the tensor core works on the other tile.  The reference
+// point m of a row only moves when the row maximum has grown by more than 2^8
+// (P stays below 256, exact enough in bf16 and harmless in the fp32 sum); only then
+// is O rescaled in tensor memory.  O is normalised by the row sum at the end and
+// rounded to bf16 once.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
@@ -22,32 +28,89 @@ namespace {
 
 using namespace ddptx;
 
-constexpr int kBlockM = 128;   // query rows per CTA
-constexpr int kBlockN = 128;   // keys per step
-constexpr int kThreads = 128;
-constexpr uint32_t kTmemCols = 256;       // S: [0,128)  O: [128,128+D)
-constexpr uint32_t kColS = 0, kColO = 128;
+constexpr int kBlockM = 128;        // query rows per tile
+constexpr int kQTiles = 2;          // query tiles per CTA
+constexpr int kBlockN = 128;        // keys per step
+constexpr int kStages = 5;          // K/V ring slots (one tile each)
+constexpr int kThreads = 384;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kLoadWarp = 8, kMmaWarp = 9;
+constexpr uint32_t kTmemCols = 512; // S_0 [0,128)  S_1 [128,256)  O_0 [256,256+D)  O_1 [256+D,256+2D)
+constexpr float kRescaleStep = 8.f; // log2 of the largest P tolerated before the reference point moves
 
-enum : unsigned { kErrWaitQ = 0x100, kErrWaitKV = 0x200, kErrWaitS = 0x300, kErrWaitO = 0x400 };
+enum : unsigned { kErrWaitQ = 0x100, kErrWaitKV = 0x200, kErrWaitS = 0x300, kErrWaitO = 0x400,
+                  kErrWaitP = 0x500, kErrWaitSlot = 0x600 };
 
 struct AttnParams {
     __nv_bfloat16 *out;
     int BH, N, D;
-    int m_blocks;
+    int m_blocks;              // CTAs per (batch, head) = ceil(N / 256)
     float scale_log2;          // scale * log2(e)
     unsigned int *status;
-    float *dbg;                // bring-up only: raw scores of the first key tile of CTA 0
 };
 
 template <int D>
 struct Smem {
-    static constexpr int kTileBytes = kBlockN * D * 2;     // one 128 x D bf16 tile
-    static constexpr int kQ = 0;
-    static constexpr int kK = kTileBytes;
-    static constexpr int kV = 2 * kTileBytes;
-    static constexpr int kBars = 3 * kTileBytes;           // 3 mbarriers + tmem slot
-    static constexpr int kTotal = kBars + 64;
+    static constexpr int kTileBytes = kBlockN * D * 2;             // one 128 x D bf16 tile
+    static constexpr int kQ = 0;                                   // two query tiles
+    static constexpr int kRing = kQTiles * kTileBytes;             // kStages K/V tiles
+    static constexpr int kBars = kRing + kStages * kTileBytes;
+    // barriers (8 bytes each): q_full, kv_full[kStages], kv_empty[kStages], s_full[2], p_full[2], o_full[2]
+    static constexpr int kNumBars = 1 + 2 * kStages + 6;
+    static constexpr int kTmemSlot = kBars + 8 * kNumBars;
+    static constexpr int kTotal = kTmemSlot + 16;
 };
+
+__device__ __forceinline__ void report(unsigned int *status, unsigned code)
+{
+    atomicCAS(status, 0u, code | (unsigned)(blockIdx.x & 0xFF));
+}
+
+// One key tile of the online softmax for one query row.  s[] holds the raw scores.
+// Returns the sum of the weights written; weights go to tensor memory as packed bf16.
+template <bool kMasked>
+__device__ __forceinline__ float row_max(const float (&s)[kBlockN], int valid)
+{
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kBlockN; i += 4) {
+        if (!kMasked || i + 0 < valid) m0 = fmaxf(m0, s[i + 0]);
+        if (!kMasked || i + 1 < valid) m1 = fmaxf(m1, s[i + 1]);
+        if (!kMasked || i + 2 < valid) m2 = fmaxf(m2, s[i + 2]);
+        if (!kMasked || i + 3 < valid) m3 = fmaxf(m3, s[i + 3]);
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+template <bool kMasked>
+__device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int valid, float c, float neg_m,
+                                                 uint32_t tmem_p)
+{
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+            const int e = h * 64 + i;
+            float p0 = ex2(fmaf(s[e], c, neg_m));
+            float p1 = ex2(fmaf(s[e + 1], c, neg_m));
+            if (kMasked) {
+                // keys past the end of the sequence get weight zero (a select, not -inf arithmetic: scale may be 0)
+                p0 = e < valid ? p0 : 0.f;
+                p1 = e + 1 < valid ? p1 : 0.f;
+            }
+            __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+            const uint32_t w = *reinterpret_cast<uint32_t *>(&b);
+            pk[i / 2] = w;
+            // the row sum takes the weights as rounded, so that O / l is an exact convex combination
+            sum0 += __uint_as_float(w << 16);
+            sum1 += __uint_as_float(w & 0xFFFF0000u);
+        }
+        tmem_st32(tmem_p + h * 32, pk);
+    }
+    return sum0 + sum1;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -57,183 +120,221 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
     // 128-byte-swizzled tiles must start on a 1024-byte boundary
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base + Smem<D>::kQ, sK = smem_base + Smem<D>::kK, sV = smem_base + Smem<D>::kV;
-    const uint32_t bar_q = smem_base + Smem<D>::kBars, bar_kv = bar_q + 8, bar_mma = bar_q + 16;
-    const uint32_t tmem_slot = bar_q + 24;
     unsigned char *smem_gen = smem_dyn + (smem_base - smem_u32(smem_dyn));
-    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + Smem<D>::kBars + 24);
+    constexpr uint32_t kTileBytes = Smem<D>::kTileBytes;
+    const uint32_t sQ = smem_base + Smem<D>::kQ, sRing = smem_base + Smem<D>::kRing;
+    const uint32_t bars = smem_base + Smem<D>::kBars;
+    const uint32_t bar_q = bars;
+    auto bar_kv_full = [&](int s) { return bars + 8u * (1 + s); };
+    auto bar_kv_empty = [&](int s) { return bars + 8u * (1 + kStages + s); };
+    auto bar_s_full = [&](int g) { return bars + 8u * (1 + 2 * kStages + g); };
+    auto bar_p_full = [&](int g) { return bars + 8u * (3 + 2 * kStages + g); };
+    auto bar_o_full = [&](int g) { return bars + 8u * (5 + 2 * kStages + g); };
+    const uint32_t tmem_slot = smem_base + Smem<D>::kTmemSlot;
+    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + Smem<D>::kTmemSlot);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x / p.m_blocks;
     const int mb = blockIdx.x - bh * p.m_blocks;
-    const int row0 = mb * kBlockM;
+    const int row0 = mb * (kQTiles * kBlockM);
     const int nkv = (p.N + kBlockN - 1) / kBlockN;
+    const int ntiles = (p.N - row0 > kBlockM) ? 2 : 1;    // query tiles of this CTA that hold rows
     constexpr int kBoxes = D / 64;                 // 64-column (128-byte) boxes per tile row
     constexpr uint32_t kBoxBytes = 128 * 128;      // 128 rows x 128 bytes
+    constexpr uint32_t kColS = 0, kColO = 256;
 
     if (tid == 0) {
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-        mbar_init(bar_q, 1); mbar_init(bar_kv, 1); mbar_init(bar_mma, 1);
+        mbar_init(bar_q, 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
+        for (int g = 0; g < kQTiles; ++g) {
+            mbar_init(bar_s_full(g), 1);
+            mbar_init(bar_p_full(g), kBlockM);
+            mbar_init(bar_o_full(g), 1);
+        }
         fence_mbar_init();
+        // a wait that expired in an earlier CTA or launch stops the rest from queueing up behind it
+        tmem_slot_gen[1] = *reinterpret_cast<volatile unsigned int *>(p.status);
     }
     if (warp == 0) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_gen;
-    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 TMEM lanes
+    const bool healthy = tmem_slot_gen[1] == 0;
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, Smem<D>::kTileBytes);
-#pragma unroll
-        for (int c = 0; c < kBoxes; ++c) tma_load_3d(sQ + c * kBoxBytes, &tm_q, bar_q, c * 64, row0, bh);
-    }
+    if (!healthy) {
+        // nothing to do
+    } else if (warp < kSoftmaxWarps) {
+        // =================================================================== softmax warpgroups
+        reg_inc<216>();
+        const int g = warp >> 2;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;   // this warp's 32 TMEM lanes
+        const uint32_t tS = tmem + lane_off + kColS + g * kBlockN;
+        const uint32_t tO = tmem + lane_off + kColO + g * D;
+        const float c = p.scale_log2;
+        float m_ref = -INFINITY, l_run = 0.f;
+        unsigned err = 0;
 
-    constexpr uint32_t kIdescS = idesc_bf16(kBlockM, kBlockN, false);
-    constexpr uint32_t kIdescO = idesc_bf16(kBlockM, D, true);
-
-    float m_run = -INFINITY, l_run = 0.f;
-    uint32_t mma_phase = 0;
-    unsigned err = 0;
-
-    for (int j = 0; j < nkv && err == 0; ++j) {
-        if (tid == 0) {
-            mbar_expect_tx(bar_kv, 2 * Smem<D>::kTileBytes);
+        if (g < ntiles) {
+            for (int j = 0; j < nkv; ++j) {
+                if (!mbar_wait(bar_s_full(g), j & 1)) { err = kErrWaitS; break; }
+                tc_fence_after();
+                float s[kBlockN];
 #pragma unroll
-            for (int c = 0; c < kBoxes; ++c) {
-                tma_load_3d(sK + c * kBoxBytes, &tm_k, bar_kv, c * 64, j * kBlockN, bh);
-                tma_load_3d(sV + c * kBoxBytes, &tm_v, bar_kv, c * 64, j * kBlockN, bh);
-            }
-        }
-        if (j == 0 && !mbar_wait(bar_q, 0)) { err = kErrWaitQ; break; }
-        if (!mbar_wait(bar_kv, j & 1)) { err = kErrWaitKV; break; }
-        __syncwarp();
-
-        // ---- S = Q K^T
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;   // 16 bf16 = 32 bytes per k-step
-                mma_ss(tmem + kColS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                       kIdescS, ks > 0);
-            }
-            mma_commit(bar_mma);
-        }
-        if (!mbar_wait(bar_mma, mma_phase)) { err = kErrWaitS; break; }
-        mma_phase ^= 1;
-        __syncwarp();
-        tc_fence_after();
-
-        // ---- online softmax on this thread's row
-        float s[kBlockN];
-#pragma unroll
-        for (int c = 0; c < kBlockN / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(lane_base + kColS + c * 32, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
-        }
-        if (p.dbg && blockIdx.x == 0 && j == 0) {
-            for (int i = 0; i < kBlockN; ++i) p.dbg[tid * kBlockN + i] = s[i];
-        }
-        const int valid = p.N - j * kBlockN;       // keys of this tile that exist
-        float mx = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < kBlockN; ++i) {
-            if (i < valid) mx = fmaxf(mx, s[i]);
-        }
-        const float m_new = fmaxf(m_run, mx * p.scale_log2);
-        const float alpha = ex2(m_run - m_new);
-        float sum = 0.f;
-        uint32_t pk[kBlockN / 2];
-#pragma unroll
-        for (int i = 0; i < kBlockN; i += 2) {
-            // keys past the end of the sequence get weight zero (no -inf arithmetic: scale may be 0)
-            const float p0 = i < valid ? ex2(fmaf(s[i], p.scale_log2, -m_new)) : 0.f;
-            const float p1 = i + 1 < valid ? ex2(fmaf(s[i + 1], p.scale_log2, -m_new)) : 0.f;
-            sum += p0 + p1;
-            __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-            pk[i / 2] = *reinterpret_cast<uint32_t *>(&h);
-        }
-        l_run = l_run * alpha + sum;
-        m_run = m_new;
-
-        // rescale this row of O
-        if (j > 0) {
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(lane_base + kColO + c * 32, r);
+                for (int cb = 0; cb < kBlockN / 32; ++cb)
+                    tmem_ld32(tS + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cb * 32]));
                 tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                tmem_st32(lane_base + kColO + c * 32, r);
-            }
-        }
-        // P (bf16, two per 32-bit column) over the first 64 columns of S
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            uint32_t r[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = pk[c * 32 + i];
-            tmem_st32(lane_base + kColS + c * 32, r);
-        }
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();
 
-        // ---- O += P V
-        if (tid == 0) {
-            tc_fence_after();
+                const int valid = p.N - j * kBlockN;       // keys of this tile that exist
+                const bool masked = valid < kBlockN;
+                const float mx = masked ? row_max<true>(s, valid) : row_max<false>(s, valid);
+                const float m_new = fmaxf(m_ref, mx * c);
+                const bool move = m_new > m_ref + kRescaleStep;   // always true on the first tile
+                if (__any_sync(0xffffffffu, move)) {
+                    const float alpha = move ? ex2(m_ref - m_new) : 1.f;
+                    if (move) m_ref = m_new;
+                    l_run *= alpha;
+                    if (j > 0) {
+                        // O_g holds the sum over tiles < j once the previous P V has completed
+                        if (!mbar_wait(bar_o_full(g), (j - 1) & 1)) { err = kErrWaitO; break; }
+                        tc_fence_after();
 #pragma unroll
-            for (int ks = 0; ks < kBlockN / 16; ++ks) {
-                // 16 keys = two 8-row groups of 1024 bytes; column blocks of 64 are one box apart
-                mma_ts(tmem + kColO, tmem + kColS + ks * 8, smem_desc_sw128(sV + ks * 2048, kBoxBytes, 1024),
-                       kIdescO, (j > 0 || ks > 0));
+                        for (int cb = 0; cb < D / 32; ++cb) {
+                            uint32_t r[32];
+                            tmem_ld32(tO + cb * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                            tmem_st32(tO + cb * 32, r);
+                        }
+                    }
+                }
+                const float sum = masked ? weights_to_tmem<true>(s, valid, c, -m_ref, tS)
+                                         : weights_to_tmem<false>(s, valid, c, -m_ref, tS);
+                l_run += sum;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar_p_full(g));
             }
-            mma_commit(bar_mma);
+            if (err == 0 && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
+            if (err == 0) {
+                // ---- epilogue: O / l -> bf16 -> global
+                tc_fence_after();
+                const int row = row0 + g * kBlockM + (warp & 3) * 32 + lane;
+                const float inv = 1.f / l_run;
+                __nv_bfloat16 *dst = p.out + ((size_t)bh * p.N + row) * D;
+#pragma unroll
+                for (int cb = 0; cb < D / 32; ++cb) {
+                    uint32_t r[32];
+                    tmem_ld32(tO + cb * 32, r);
+                    tmem_wait_ld();
+                    if (row < p.N) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * h]) * inv,
+                                                                         __uint_as_float(r[i + 2 * h + 1]) * inv);
+                                w[h] = *reinterpret_cast<uint32_t *>(&v);
+                            }
+                            *reinterpret_cast<uint4 *>(dst + cb * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+            } else {
+                report(p.status, err);
+            }
         }
-        if (!mbar_wait(bar_mma, mma_phase)) { err = kErrWaitO; break; }
-        mma_phase ^= 1;
-        __syncwarp();
-        tc_fence_after();
+    } else {
+        reg_dec<72>();
+        if (warp == kLoadWarp && lane == 0) {
+            // =============================================================== TMA producer
+            mbar_expect_tx(bar_q, ntiles * kTileBytes);
+            for (int g = 0; g < ntiles; ++g)
+#pragma unroll
+                for (int cx = 0; cx < kBoxes; ++cx)
+                    tma_load_3d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q, cx * 64, row0 + g * kBlockM, bh);
+            // ring items: 2j = K tile j, 2j+1 = V tile j
+            for (int item = 0; item < 2 * nkv; ++item) {
+                const int slot = item % kStages, use = item / kStages;
+                if (use > 0 && !mbar_wait(bar_kv_empty(slot), (use - 1) & 1)) { report(p.status, kErrWaitSlot); break; }
+                const uint32_t dst = sRing + slot * kTileBytes;
+                const CUtensorMap *tm = (item & 1) ? &tm_v : &tm_k;
+                mbar_expect_tx(bar_kv_full(slot), kTileBytes);
+#pragma unroll
+                for (int cx = 0; cx < kBoxes; ++cx)
+                    tma_load_3d(dst + cx * kBoxBytes, tm, bar_kv_full(slot), cx * 64, (item >> 1) * kBlockN, bh);
+            }
+        } else if (warp == kMmaWarp && lane == 0) {
+            // =============================================================== MMA issuer
+            constexpr uint32_t kIdescS = idesc_bf16(kBlockM, kBlockN, false);
+            constexpr uint32_t kIdescO = idesc_bf16(kBlockM, D, true);
+            unsigned err = 0;
+            // S_g = Q_g K^T for the K tile in `slot`
+            auto issue_s = [&](int g, int slot) {
+                const uint32_t a = sQ + g * kTileBytes, b = sRing + slot * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;   // 16 bf16 = 32 bytes per k-step
+                    mma_ss(tmem + kColS + g * kBlockN, smem_desc_sw128(a + off, 16, 1024),
+                           smem_desc_sw128(b + off, 16, 1024), kIdescS, ks > 0);
+                }
+                mma_commit(bar_s_full(g));
+            };
+            // O_g (+)= P_g V for the V tile in `slot`
+            auto issue_o = [&](int g, int slot, bool first) {
+                const uint32_t b = sRing + slot * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < kBlockN / 16; ++ks) {
+                    // 16 keys = two 8-row groups of 1024 bytes; column blocks of 64 are one box apart
+                    mma_ts(tmem + kColO + g * D, tmem + kColS + g * kBlockN + ks * 8,
+                           smem_desc_sw128(b + ks * 2048, kBoxBytes, 1024), kIdescO, (!first || ks > 0));
+                }
+                mma_commit(bar_o_full(g));
+            };
+            auto wait_item = [&](int item) {
+                return mbar_wait(bar_kv_full(item % kStages), (item / kStages) & 1);
+            };
+            do {
+                if (!mbar_wait(bar_q, 0)) { err = kErrWaitQ; break; }
+                if (!wait_item(0)) { err = kErrWaitKV; break; }
+                tc_fence_after();
+                for (int g = 0; g < ntiles; ++g) issue_s(g, 0);
+                mma_commit(bar_kv_empty(0));
+                for (int j = 0; j < nkv && err == 0; ++j) {
+                    const int item_v = 2 * j + 1, item_k = 2 * j + 2;
+                    const bool more = j + 1 < nkv;
+                    if (!wait_item(item_v)) { err = kErrWaitKV; break; }
+                    for (int g = 0; g < ntiles; ++g) {
+                        if (!mbar_wait(bar_p_full(g), j & 1)) { err = kErrWaitP; break; }
+                        tc_fence_after();
+                        issue_o(g, item_v % kStages, j == 0);
+                        if (more) {
+                            if (g == 0 && !wait_item(item_k)) { err = kErrWaitKV; break; }
+                            tc_fence_after();
+                            issue_s(g, item_k % kStages);
+                        }
+                    }
+                    if (err) break;
+                    mma_commit(bar_kv_empty(item_v % kStages));
+                    if (more) mma_commit(bar_kv_empty(item_k % kStages));
+                }
+            } while (false);
+            if (err) report(p.status, err);
+        }
     }
 
     __syncwarp();
-    if (err != 0) {
-        atomicCAS(p.status, 0u, err | (unsigned)(blockIdx.x & 0xFF));
-        // give copies that may still be in flight time to land before the shared memory is released
+    if (*reinterpret_cast<volatile unsigned int *>(p.status) != 0) {
+        // a wait expired somewhere: give copies that may still be in flight time to land before the
+        // shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-    } else {
-        // ---- epilogue: O / l -> bf16 -> global
-        const int row = row0 + tid;
-        const float inv = 1.f / l_run;
-        __nv_bfloat16 *dst = p.out + ((size_t)bh * p.N + row) * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(lane_base + kColO + c * 32, r);
-            tmem_wait_ld();
-            if (row < p.N) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int h = 0; h < 4; ++h) {
-                        __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * h]) * inv,
-                                                                 __uint_as_float(r[i + 2 * h + 1]) * inv);
-                        w[h] = *reinterpret_cast<uint32_t *>(&v);
-                    }
-                    *reinterpret_cast<uint4 *>(dst + c * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-            }
-        }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 0) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
 // ---------------------------------------------------------------------------
@@ -290,7 +391,7 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
 }
 
 int attention_impl(const void *q, const void *k, const void *v, void *out, int B, int H, int N, int D,
-                   float scale, void *stream, float *dbg)
+                   float scale, void *stream)
 {
     if (!q || !k || !v || !out) return DD_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || N <= 0 || D <= 0) return DD_ERR_INVALID_ARG;
@@ -299,7 +400,7 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     if (D != 64 && D != 128) return DD_ERR_UNSUPPORTED;
     if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) != 0) return DD_ERR_UNSUPPORTED;
     const long BH = (long)B * H;
-    const int m_blocks = (N + kBlockM - 1) / kBlockM;
+    const int m_blocks = (N + kQTiles * kBlockM - 1) / (kQTiles * kBlockM);
     if (BH * m_blocks >= (1L << 31) || BH >= (1L << 31)) return DD_ERR_UNSUPPORTED;
 
     dd::DeviceCtx *ctx = dd::current_ctx();
@@ -320,7 +421,6 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     p.m_blocks = m_blocks;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->attn_status;
-    p.dbg = dbg;
     cudaStream_t s = (cudaStream_t)stream;
     return D == 64 ? launch<64>(tq, tk, tv, p, s) : launch<128>(tq, tk, tv, p, s);
 }
@@ -330,13 +430,5 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
 extern "C" int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
                                   int B, int H, int N, int D, float scale, void *stream)
 {
-    return attention_impl(q, k, v, out, B, H, N, D, scale, stream, nullptr);
-}
-
-// Bring-up aid (not part of the public header): also dumps the raw fp32 scores
-// S = Q K^T of the first key tile of the first CTA into dbg[128*128].
-extern "C" int dd_debug_attention(const void *q, const void *k, const void *v, void *out,
-                                  int B, int H, int N, int D, float scale, void *stream, float *dbg)
-{
-    return attention_impl(q, k, v, out, B, H, N, D, scale, stream, dbg);
+    return attention_impl(q, k, v, out, B, H, N, D, scale, stream);
 }
