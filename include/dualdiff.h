@@ -96,7 +96,7 @@ int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
  * drafter_logits, verifier_logits: [B,P,V] bf16 (drafter_logits may be NULL
  * unless the mode is KL); tokens int32 [B,P]; mask_flags uint8 [B,P];
  * out_tokens int32 [B,P] (may alias tokens); out_mask uint8 [B,P]; out_score
- * fp32 [B,P], nullable.  The 16-byte vector path needs V % 8 == 0 and 16-byte
+ * fp32 [B,P], nullable.  The streaming path needs V % 8 == 0 and 16-byte
  * aligned logits; otherwise a slower element-wise path is taken.
  * Supported: P <= 8192; V < 2^31 / 2.
  * Errors: DD_ERR_INVALID_ARG (null required pointer, B/P/V <= 0, k < 0, unknown
@@ -131,9 +131,9 @@ int dd_verify_host(const void *drafter_logits, const void *verifier_logits,
  * cudaMalloc/cudaFree, or that does not own the allocator of its process: this
  * call performs no cudaMalloc, cudaFree or other allocating routine.  Its scratch
  * (chunk partials, row results, completion counters) is a fixed array of about
- * 2.1 MB inside the library, held by every GPU that loads the library until the
+ * 4.3 MB inside the library, held by every GPU that loads the library until the
  * process exits.
- * Limits: B*P <= 4096 and B*P*ceil(V/8192) <= 65536; larger problems return
+ * Limits: B*P <= 4096 and B*P*ceil(V/4096) <= 131072; larger problems return
  * DD_ERR_UNSUPPORTED and launch nothing.
  * The first call on each device looks up the array's device address; make that
  * first call outside any stream capture.  All calls on a device share the one
@@ -157,6 +157,14 @@ size_t dd_verify_workspace_bytes(int B, int P, int V);
  * the device.  Returns DD_OK / DD_ERR_TIMEOUT / DD_ERR_CUDA.
  */
 int dd_attention_status(void);
+
+/*
+ * Device-side health word of dd_verify for the current device, with the same
+ * meaning and return values as dd_attention_status: non-zero once a bounded wait
+ * for a shared-memory copy or queue has expired (the outputs of that call are
+ * undefined; dd_release() returns the scratch to its initial state).
+ */
+int dd_verify_status(void);
 
 /* Number of kernels launched by this library in this process (all devices). */
 uint64_t dd_launch_count(void);

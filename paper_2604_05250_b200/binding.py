@@ -21,7 +21,7 @@ DD_FLAG_PROBABILISTIC, DD_FLAG_EMIT_DRAFTER = 0x100, 0x200
 # every symbol include/dualdiff.h declares
 EXPORTS = (
     "dd_bidir_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
-    "dd_verify_workspace_bytes", "dd_attention_status", "dd_launch_count", "dd_release",
+    "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
     "dd_status_string", "dd_last_cuda_error", "dd_version",
 )
 
@@ -54,9 +54,10 @@ def lib() -> ctypes.CDLL:
         L.dd_verify_static.argtypes = ver
         L.dd_verify_static.restype = i32
         for name in ("dd_bidir_attention", "dd_bidir_attention_host", "dd_verify", "dd_verify_host",
-                     "dd_attention_status", "dd_release", "dd_version"):
+                     "dd_attention_status", "dd_verify_status", "dd_release", "dd_version"):
             getattr(L, name).restype = i32
         L.dd_attention_status.argtypes = []
+        L.dd_verify_status.argtypes = []
         L.dd_release.argtypes = []
         L.dd_version.argtypes = []
         L.dd_verify_workspace_bytes.argtypes = [i32, i32, i32]
@@ -155,6 +156,10 @@ def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, se
 
 def attention_status() -> int:
     return int(lib().dd_attention_status())
+
+
+def verify_status() -> int:
+    return int(lib().dd_verify_status())
 
 
 def launch_count() -> int:

@@ -25,6 +25,8 @@ int cuda_fail(cudaError_t e, const char *where)
     return DD_ERR_CUDA;
 }
 
+void set_error_text(const char *text) { snprintf(g_err, sizeof g_err, "%s", text); }
+
 void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 DeviceCtx *current_ctx(int *device_out)

@@ -31,6 +31,9 @@ int ensure_bytes(void **ptr, size_t *have, size_t need);
 // Records a CUDA error text for dd_last_cuda_error() and returns DD_ERR_CUDA.
 int cuda_fail(cudaError_t e, const char *where);
 
+// Sets the text dd_last_cuda_error() returns.
+void set_error_text(const char *text);
+
 void count_launch(unsigned n = 1);
 
 #define DD_CUDA_TRY(expr)                                         \

@@ -1,0 +1,271 @@
+// Decision stage, row fold and partial publication of dd_verify (warp-level code).
+// Included by dd_verify_common.cuh.
+#pragma once
+
+namespace ddv {
+
+// ---------------------------------------------------------------------------
+// Decision stage for one sequence, run by one warp (the one that completed it).
+//
+// Minimum-keep top-k without sorting: the k-th largest reliability t among the flagged
+// positions is found by a bitwise binary search on the order-preserving integer image of
+// the score; positions above t are kept, and those equal to t are kept lowest index first
+// until k are kept in all.  This equals ranking by (reliability descending, index ascending).
+//
+// Lane l owns positions l, l+32, l+64, ...  With R > 0 their keys stay in registers
+// (P <= 32 R); with R == 0 they are re-read from memory on every pass (any P).
+// The parameters come by value: only this rare call copies them to the stack.
+template <int R>
+__device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned full = 0xFFFFFFFFu;
+    const long base = (long)b * p.P;
+    const bool kl_mode = p.algo == DD_MODE_KL;
+    const int nk = (p.P + 31) / 32;                 // positions per lane (upper bound)
+    constexpr int kRegs = R > 0 ? R : 1;
+
+    // key of position i: order-preserving image of its reliability, 0 outside the set.
+    // Both loads are unconditional (the score slot exists for every position), so a pass
+    // over the keys is a batch of independent loads.
+    auto load_key = [&](int i) -> uint32_t {
+        const int ic = min(i, p.P - 1);
+        const uint8_t f = p.flags[base + ic];
+        const float s = __ldcg(p.row_score + base + ic);
+        return (i < p.P && f) ? orderable(kl_mode ? 0.0f - s : s) : 0u;
+    };
+    uint32_t key_reg[kRegs];
+    if (R > 0) {
+#pragma unroll
+        for (int r = 0; r < kRegs; ++r) key_reg[r] = r < nk ? load_key(lane + 32 * r) : 0u;
+    }
+    // f(r, key) for every position lane + 32 r of this lane, r ascending (uniform trip count)
+    auto for_each_key = [&](auto f) {
+        if (R > 0) {
+#pragma unroll
+            for (int r = 0; r < kRegs; ++r)
+                if (r < nk) f(r, key_reg[r]);
+        } else {
+            for (int r = 0; r < nk; ++r) f(r, load_key(lane + 32 * r));
+        }
+    };
+    auto score_of = [&](uint32_t key) -> float {     // inverse of the key map (key != 0)
+        const float rel = __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
+        return kl_mode ? 0.0f - rel : rel;
+    };
+    // number of keys of the whole sequence with key >= cand, or key > cand
+    auto count_keys = [&](uint32_t cand, bool strictly) -> int {
+        int cnt = 0;
+        if (R > 0) {
+#pragma unroll
+            for (int r = 0; r < kRegs; ++r) cnt += strictly ? (key_reg[r] > cand) : (key_reg[r] >= cand);
+        } else {
+#pragma unroll 8
+            for (int r = 0; r < nk; ++r) {
+                const uint32_t k = load_key(lane + 32 * r);
+                cnt += strictly ? (k > cand) : (k >= cand);
+            }
+        }
+        return __reduce_add_sync(full, cnt);
+    };
+
+    // Eq. 6 normaliser: sum of KL over the drafter-decoded set, in a fixed order
+    const int n_flagged = count_keys(0u, true);
+    double kl_sum = 0.0;
+    if (kl_mode && p.probabilistic) {
+        double part = 0.0;
+        for_each_key([&](int, uint32_t k) { if (k) part += (double)score_of(k); });
+        kl_sum = warp_sum(part);
+    }
+    auto fails = [&](int i, float s) -> bool {
+        if (p.algo == DD_MODE_TRUST) return false;
+        if (!p.probabilistic) return kl_mode ? (s > p.tau) : (s < p.tau);
+        const uint32_t w = philox_first_word((uint32_t)i, (uint32_t)b, p.seed_lo, p.seed_hi);
+        const double u = (double)(w >> 8) * (1.0 / 16777216.0);
+        const double prob = kl_mode ? (kl_sum > 0.0 ? (double)s / kl_sum : 0.0) : 1.0 - (double)s;
+        return u < prob;
+    };
+
+    // which of this lane's positions fail (bit r), for up to 32 positions per lane; beyond that
+    // (R == 0 with P > 1024) the rule is evaluated again where it is needed
+    unsigned fail_bits = 0u;
+    bool any_fail = false;
+    for_each_key([&](int r, uint32_t k) {
+        const bool f = k != 0u && fails(lane + 32 * r, score_of(k));
+        any_fail |= f;
+        if (r < 32 && f) fail_bits |= 1u << r;
+    });
+    any_fail = __any_sync(full, any_fail);
+
+    // top-k threshold, needed only if some position fails and fewer than all are protected
+    uint32_t thr = 0u;          // k-th largest key
+    int quota = 0;              // how many of the positions equal to thr are still kept
+    bool topk_active = false, keep_all = false;
+    if (p.k > 0 && any_fail) {
+        if (n_flagged <= p.k) {
+            keep_all = true;
+        } else {
+            topk_active = true;
+            for (int bit = 31; bit >= 0; --bit) {
+                const uint32_t cand = thr | (1u << bit);
+                if (count_keys(cand, false) >= p.k) thr = cand;
+            }
+            quota = p.k - count_keys(thr, true);
+        }
+    }
+
+    int equal_seen = 0;         // positions equal to thr at lower indices
+    for_each_key([&](int r, uint32_t key) {
+        const int i = lane + 32 * r;
+        const long t = base + i;
+        const bool flagged = key != 0u;
+        bool protect = keep_all;
+        if (topk_active) {
+            const bool eq = flagged && key == thr;
+            const unsigned eq_mask = __ballot_sync(full, eq);
+            const int my_rank = equal_seen + __popc(eq_mask & ((1u << lane) - 1u));
+            equal_seen += __popc(eq_mask);
+            protect = key > thr || (eq && my_rank < quota);
+        }
+        if (i >= p.P) return;
+        const int32_t tok = p.tokens[t];
+        if (!flagged) {
+            p.out_tokens[t] = tok;
+            p.out_mask[t] = 0;
+            if (p.out_score) p.out_score[t] = 0.0f;
+            return;
+        }
+        const float s = __ldcg(p.row_score + t);
+        const bool failed = r < 32 ? ((fail_bits >> r) & 1u) != 0u : fails(i, s);
+        const bool remask = failed && !protect;
+        p.out_mask[t] = remask ? 1 : 0;
+        p.out_tokens[t] = (remask || p.emit_drafter) ? tok : __ldcg(p.row_argmax + t);
+        if (p.out_score) p.out_score[t] = s;
+    });
+}
+
+__device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b)
+{
+    if (p.P <= 256) decide_sequence_impl<8>(p, b);
+    else if (p.P <= 1024) decide_sequence_impl<32>(p, b);
+    else decide_sequence_impl<0>(p, b);
+}
+
+// One sequence has one more completed row; the warp that completes the sequence decides it.
+__device__ __forceinline__ void row_done(const VerifyParams &p, int b)
+{
+    const int lane = threadIdx.x & 31;
+    int last = 0;
+    if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(p.seq_counter + b, 1u) == (unsigned)(p.P - 1);
+    }
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
+    __threadfence();
+    if (lane == 0) p.seq_counter[b] = 0u;      // ready for the next launch
+    decide_sequence(p, b);
+}
+
+// The calling warp saw the row's last chunk published: fold the row's partials in chunk
+// order (fp64), store the row's score and argmax, and report the row to its sequence.
+template <bool KL>
+__device__ __forceinline__ void fold_row(const VerifyParams &p, int row)
+{
+    const int lane = threadIdx.x & 31;
+    __threadfence();
+    const Partial *src = p.partials + (size_t)row * p.nchunks;
+    float bm_v = -INFINITY, bm_d = -INFINITY;
+    int bidx = 0x7FFFFFFF;
+    for (int ch = lane; ch < p.nchunks; ch += 32) {
+        const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + ch));
+        const float mv = a.x, md = a.w;
+        const int ix = __float_as_int(a.z);
+        if (mv > bm_v || (mv == bm_v && ix < bidx)) { bm_v = mv; bidx = ix; }
+        bm_d = fmaxf(bm_d, md);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xFFFFFFFFu, bm_v, o);
+        const int oi = __shfl_xor_sync(0xFFFFFFFFu, bidx, o);
+        if (om > bm_v || (om == bm_v && oi < bidx)) { bm_v = om; bidx = oi; }
+        bm_d = fmaxf(bm_d, __shfl_xor_sync(0xFFFFFFFFu, bm_d, o));
+    }
+    const float Mv = bm_v * kLog2e, Md = bm_d * kLog2e;
+    double sv = 0.0, sd = 0.0, tt = 0.0;
+    for (int ch = lane; ch < p.nchunks; ch += 32) {
+        const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + ch));
+        const float4 bq = __ldcg(reinterpret_cast<const float4 *>(src + ch) + 1);
+        sv += (double)a.y * exp2((double)(a.x * kLog2e) - (double)Mv);
+        if (KL) {
+            const double f = exp2((double)(a.w * kLog2e) - (double)Md);
+            sd += (double)bq.x * f;
+            tt += (double)bq.y * f;
+        }
+    }
+    sv = warp_sum(sv);
+    if (KL) { sd = warp_sum(sd); tt = warp_sum(tt); }
+    if (lane == 0) {
+        float score;
+        if (KL) {
+            const double lse_v = (double)Mv * kLn2 + log(sv);
+            const double lse_d = (double)Md * kLn2 + log(sd);
+            const double kl = tt / sd - lse_d + lse_v;
+            score = (float)fmax(kl, 0.0);
+        } else {
+            // the maximum's own term is 2^(m*log2e - M), not exactly 1
+            score = (float)(exp2((double)bm_v * (double)kLog2e - (double)Mv) / sv);
+        }
+        __stcg(p.row_score + row, score);
+        __stcg(p.row_argmax + row, bidx);
+        p.row_counter[row] = 0u;      // ready for the next launch
+    }
+    __syncwarp();
+    row_done(p, row / p.P);
+}
+
+// Publishes up to 32 finished (row, chunk) partials at once -- lane l holds entry l, its row in
+// pad0 and its chunk in pad1 (as integer bits) -- with one fence for the whole batch; the rows
+// whose last chunk was among them are then folded one after the other.  An entry with a
+// negative chunk stands for an unflagged row, which is only reported to its sequence.
+template <bool KL>
+__device__ __forceinline__ void publish_batch(const VerifyParams &p, const Partial &c, int n)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned full = 0xFFFFFFFFu;
+    const int row = __float_as_int(c.pad0), chunk = __float_as_int(c.pad1);
+    const bool mine = lane < n;
+    if (mine && chunk >= 0) {
+        Partial *dst = p.partials + (size_t)row * p.nchunks + chunk;
+        const float4 a = make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d);
+        const float4 bq = make_float4(c.s_d, c.t, 0.f, 0.f);
+        __stcg(reinterpret_cast<float4 *>(dst), a);
+        __stcg(reinterpret_cast<float4 *>(dst) + 1, bq);
+    }
+    __threadfence();
+    bool last = false;
+    if (mine && chunk >= 0) last = atomicAdd(p.row_counter + row, 1u) == (unsigned)(p.nchunks - 1);
+    unsigned todo = __ballot_sync(full, last);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        fold_row<KL>(p, __shfl_sync(full, row, src));
+    }
+    todo = __ballot_sync(full, mine && chunk < 0);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        row_done(p, __shfl_sync(full, row, src) / p.P);
+    }
+}
+
+// One partial, held by every lane alike.
+template <bool KL>
+__device__ __forceinline__ void chunk_done(const VerifyParams &p, int row, int chunk, Partial c)
+{
+    c.pad0 = __int_as_float(row);
+    c.pad1 = __int_as_float(chunk);
+    publish_batch<KL>(p, c, 1);
+}
+
+}  // namespace ddv

@@ -1,0 +1,273 @@
+// Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
+//
+// One persistent CTA per SM: fifteen warps stream, one warp publishes.  A streaming
+// warp takes a (row, chunk) of 4096 logits from the CTA's queue and pulls it through
+// its private ring of three shared-memory stages in pieces of 1024 logits per tensor
+// with bulk asynchronous copies (cp.async.bulk + mbarrier), so loads stay in flight
+// while the warp computes.  Within a chunk every lane keeps its own running maxima,
+// reference points and sums (packed bf16x2 maxima, packed fp32 pairs); lanes talk to
+// each other only when the chunk ends.  The finished partial goes into a
+// shared-memory queue; the publishing warp drains it in batches (one fence per batch),
+// counts chunks per row, folds completed rows and decides completed sequences, so the
+// streaming warps never wait for a round trip to global memory.  No CTA-wide barrier
+// follows start-up.
+#pragma once
+
+#include "dd_verify_common.cuh"
+
+namespace ddv {
+
+constexpr int kSStreamWarps = 15;                             // warps that stream
+constexpr int kSWarps = kSStreamWarps + 1;                    // + one that publishes finished chunks
+constexpr int kSThreads = kSWarps * 32;
+constexpr int kSQueue = 64;                                   // finished-chunk queue slots
+constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits: one ring stage per tensor
+constexpr int kPiecesPerChunk = 4;
+constexpr int kSChunk = kPiece * kPiecesPerChunk;             // 4096 logits per (row, chunk)
+constexpr int kSStages = 3;
+constexpr unsigned kErrWaitPiece = 0x700, kErrWaitQueue = 0x800;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *ptr)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Untiled bulk copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+
+// Packed fp32 pairs (one instruction works on two values).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+struct PieceDesc {     // what a ring stage holds; row < 0: nothing more will come
+    int row, chunk, e_begin, n;
+    int ordinal, last, pad0, pad1;   // ordinal: piece number within its chunk
+};
+
+// Running state of one lane over the pieces of a chunk.
+struct LaneState {
+    uint32_t max2_v, max2_d;   // packed bf16x2 running maxima (even / odd logits of the lane's words)
+    uint32_t where2_v;         // per half: ordinal of the word that first attained the verifier's maximum
+    float M_v, M_d;            // reference points: lane maximum * log2e
+    unsigned long long s_v, s_d, t;   // packed fp32 pairs (even / odd logits)
+};
+
+__device__ __forceinline__ void lane_reset(LaneState &L)
+{
+    L.max2_v = L.max2_d = 0xFF80FF80u;     // -inf, -inf
+    L.where2_v = 0u;
+    L.M_v = L.M_d = -INFINITY;
+    L.s_v = L.s_d = L.t = 0ull;
+}
+
+// One piece (n logits, a multiple of 8; lane's vector j covers logits (lane + 32 j) * 8 ..+7).
+template <bool KL>
+__device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecPerThread],
+                                           const uint4 (&rd)[kVecPerThread], int n, int lane, int ordinal)
+{
+    // pass 1: packed running maxima; the word ordinal (within this piece) where a half first rose
+    uint32_t max2_v = L.max2_v, max2_d = L.max2_d, where2 = 0u;
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        const uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
+        const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const __nv_bfloat162 w = *reinterpret_cast<const __nv_bfloat162 *>(&wv[h]);
+            const __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162 *>(&max2_v);
+            const uint32_t rose = __hgt2_mask(w, m);                  // 0xFFFF per half that rises
+            const __nv_bfloat162 m_new = __hmax2(m, w);
+            max2_v = *reinterpret_cast<const uint32_t *>(&m_new);
+            const uint32_t q2 = (uint32_t)(j * 4 + h) * 0x00010001u;
+            where2 = (where2 & ~rose) | (q2 & rose);
+            if (KL) {
+                const __nv_bfloat162 d = *reinterpret_cast<const __nv_bfloat162 *>(&wd[h]);
+                const __nv_bfloat162 md = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&max2_d), d);
+                max2_d = *reinterpret_cast<const uint32_t *>(&md);
+            }
+        }
+    }
+    {
+        // halves that rose during this piece take (piece ordinal, word ordinal)
+        const __nv_bfloat162 before = *reinterpret_cast<const __nv_bfloat162 *>(&L.max2_v);
+        const __nv_bfloat162 after = *reinterpret_cast<const __nv_bfloat162 *>(&max2_v);
+        const uint32_t rose = __hgt2_mask(after, before);
+        const uint32_t q2 = where2 + (uint32_t)(ordinal * 16) * 0x00010001u;
+        L.where2_v = (L.where2_v & ~rose) | (q2 & rose);
+        L.max2_v = max2_v;
+        L.max2_d = max2_d;
+    }
+    // move the reference points; the sums follow
+    const float M_v = fmaxf(bf16lo(max2_v), bf16hi(max2_v)) * kLog2e;
+    {
+        const float f = rescale_factor(L.M_v, M_v);
+        L.s_v = fma2(L.s_v, pack2(f, f), 0ull);
+        L.M_v = M_v;
+    }
+    float M_d = 0.f;
+    if (KL) {
+        M_d = fmaxf(bf16lo(max2_d), bf16hi(max2_d)) * kLog2e;
+        const float f = rescale_factor(L.M_d, M_d);
+        const unsigned long long f2 = pack2(f, f);
+        L.s_d = fma2(L.s_d, f2, 0ull);
+        L.t = fma2(L.t, f2, 0ull);
+        L.M_d = M_d;
+    }
+    // pass 2: one ex2 per logit against the lane's reference
+    const unsigned long long log2e2 = pack2(kLog2e, kLog2e);
+    const unsigned long long nMv2 = pack2(-M_v, -M_v), nMd2 = pack2(-M_d, -M_d);
+    const unsigned long long neg1 = pack2(-1.f, -1.f);
+    unsigned long long s_v = L.s_v, s_d = L.s_d, t = L.t;
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        if ((lane + j * 32) * 8 < n) {
+            const uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
+            const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const unsigned long long v2 = pack2(bf16lo(wv[h]), bf16hi(wv[h]));
+                float a0, a1;
+                unpack2(fma2(v2, log2e2, nMv2), a0, a1);
+                s_v = add2(s_v, pack2(ex2_approx(a0), ex2_approx(a1)));
+                if (KL) {
+                    const unsigned long long d2 = pack2(bf16lo(wd[h]), bf16hi(wd[h]));
+                    float b0, b1;
+                    unpack2(fma2(d2, log2e2, nMd2), b0, b1);
+                    const unsigned long long e2 = pack2(ex2_approx(b0), ex2_approx(b1));
+                    s_d = add2(s_d, e2);
+                    t = fma2(e2, fma2(v2, neg1, d2), t);          // e * (d - v)
+                }
+            }
+        }
+    }
+    L.s_v = s_v; L.s_d = s_d; L.t = t;
+}
+
+// The chunk has ended: the 32 lane states become one partial (lane 0's copy is the one used).
+template <bool KL>
+__device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chunk_begin, int lane)
+{
+    const unsigned full = 0xFFFFFFFFu;
+    Partial c;
+    const float lo_m = bf16lo(L.max2_v), hi_m = bf16hi(L.max2_v);
+    auto element_of = [&](uint32_t q, int odd) {     // q = piece * 16 + j * 4 + h
+        return chunk_begin + (int)(q >> 4) * kPiece + (lane + 32 * (int)((q >> 2) & 3u)) * 8 +
+               2 * (int)(q & 3u) + odd;
+    };
+    const int e_lo = element_of(L.where2_v & 0xFFFFu, 0), e_hi = element_of(L.where2_v >> 16, 1);
+    c.m_v = fmaxf(lo_m, hi_m);
+    c.idx = lo_m > hi_m ? e_lo : (hi_m > lo_m ? e_hi : min(e_lo, e_hi));
+    float a0, a1;
+    unpack2(L.s_v, a0, a1);
+    c.s_v = a0 + a1;
+    c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f;
+    if (KL) {
+        c.m_d = fmaxf(bf16lo(L.max2_d), bf16hi(L.max2_d));
+        unpack2(L.s_d, a0, a1);
+        c.s_d = a0 + a1;
+        unpack2(L.t, a0, a1);
+        c.t = a0 + a1;
+    }
+    c.pad0 = c.pad1 = 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial other;
+        other.m_v = __shfl_xor_sync(full, c.m_v, o);
+        other.s_v = __shfl_xor_sync(full, c.s_v, o);
+        other.idx = __shfl_xor_sync(full, c.idx, o);
+        other.m_d = 0.f; other.s_d = 0.f; other.t = 0.f;
+        if (KL) {
+            other.m_d = __shfl_xor_sync(full, c.m_d, o);
+            other.s_d = __shfl_xor_sync(full, c.s_d, o);
+            other.t = __shfl_xor_sync(full, c.t, o);
+        }
+        // both lanes of a pair merge (lower lane's, upper lane's) in that order: same bits in both
+        if ((lane & o) == 0) {
+            merge_partial<KL>(c, other);
+        } else {
+            merge_partial<KL>(other, c);
+            c.m_v = other.m_v; c.s_v = other.s_v; c.idx = other.idx;
+            c.m_d = other.m_d; c.s_d = other.s_d; c.t = other.t;
+        }
+    }
+    return c;
+}
+
+// Queue of finished chunks between the streaming warps (many producers) and the publishing
+// warp (one consumer), in shared memory.
+struct ChunkQueue {
+    Partial entry[kSQueue];
+    unsigned int ready[kSQueue];     // sequence number + 1 of the entry the slot holds
+    unsigned int tail;               // next sequence number to hand out
+    unsigned int head;               // entries below this have been taken
+    unsigned int done;               // streaming warps that have finished
+    unsigned int pad;
+};
+
+// One lane of a streaming warp hands over an entry.  False if the queue stayed full.
+__device__ __forceinline__ bool queue_push(ChunkQueue &q, const Partial &e)
+{
+    const unsigned int seq = atomicAdd(&q.tail, 1u);
+    volatile unsigned int *head = &q.head;
+    unsigned it = 0;
+    while (seq - *head >= (unsigned)kSQueue) {
+        if (++it > (1u << 22)) return false;
+        __nanosleep(64);
+    }
+    q.entry[seq % kSQueue] = e;
+    __threadfence_block();
+    *(volatile unsigned int *)&q.ready[seq % kSQueue] = seq + 1u;
+    return true;
+}
+
+}  // namespace ddv
+
+#include "dd_verify_stream_kernel.cuh"
