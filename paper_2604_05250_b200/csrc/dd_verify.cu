@@ -143,6 +143,7 @@ template <bool KL>
 __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const VerifyParams p)
 {
     __shared__ Partial warp_part[kWarps];
+    __shared__ DecideStage s_decide;                // decision stage (warp 0 only)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x / p.nchunks;
@@ -150,7 +151,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
 
     if (!p.flags[row]) {
         // Unflagged rows cost nothing; warp 0 of their chunk-0 CTA reports the row as complete.
-        if (chunk == 0 && warp == 0) row_done(p, row / p.P);
+        if (chunk == 0 && warp == 0) row_done(p, row / p.P, &s_decide);
         return;
     }
     const int e_begin = chunk * p.chunk;
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
     Partial c = warp_part[0];
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) merge_partial<KL>(c, warp_part[w]);
-    chunk_done<KL>(p, row, chunk, c);
+    chunk_done<KL>(p, row, chunk, c, &s_decide);
 }
 
 // ---------------------------------------------------------------------------

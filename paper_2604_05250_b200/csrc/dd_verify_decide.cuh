@@ -12,18 +12,28 @@ namespace ddv {
 // the score; positions above t are kept, and those equal to t are kept lowest index first
 // until k are kept in all.  This equals ranking by (reliability descending, index ascending).
 //
-// Lane l owns positions l, l+32, l+64, ...  With R > 0 their keys stay in registers
-// (P <= 32 R); with R == 0 they are re-read from memory on every pass (any P).
-// The parameters come by value: only this rare call copies them to the stack.
-template <int R>
-__device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
+// Lane l owns positions l, l+32, l+64, ...  The keys of a sequence of up to kDecideKeys
+// positions, with their tokens and argmaxes, are staged in the caller's shared memory; longer sequences re-read
+// them from memory on every pass.  The code runs once per sequence, from a cold instruction
+// cache: it is written as short loops, not unrolled.
+// The parameters come by value: only this rare call copies them to the stack.  dry: every
+// load and every step, but no store.
+constexpr int kDecideKeys = 1024;
+
+struct __align__(16) DecideStage {      // one per deciding warp, in shared memory
+    uint32_t key[kDecideKeys];
+    int32_t tok[kDecideKeys];      // tokens[b, i]
+    int32_t top[kDecideKeys];      // verifier argmax of position i
+};
+
+__device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b, DecideStage *stage, bool dry)
 {
     const int lane = threadIdx.x & 31;
     const unsigned full = 0xFFFFFFFFu;
     const long base = (long)b * p.P;
     const bool kl_mode = p.algo == DD_MODE_KL;
     const int nk = (p.P + 31) / 32;                 // positions per lane (upper bound)
-    constexpr int kRegs = R > 0 ? R : 1;
+    const bool staged = p.P <= kDecideKeys;
 
     // key of position i: order-preserving image of its reliability, 0 outside the set.
     // Both loads are unconditional (the score slot exists for every position), so a pass
@@ -34,39 +44,54 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
         const float s = __ldcg(p.row_score + base + ic);
         return (i < p.P && f) ? orderable(kl_mode ? 0.0f - s : s) : 0u;
     };
-    uint32_t key_reg[kRegs];
-    if (R > 0) {
+    if (staged) {
+        // eight positions per lane at a time: every load of the group first (independent, so
+        // they overlap), then the stores
+        for (int r0 = 0; r0 < nk; r0 += 8) {
+            uint32_t k[8];
+            int32_t tk[8], tp[8];
 #pragma unroll
-        for (int r = 0; r < kRegs; ++r) key_reg[r] = r < nk ? load_key(lane + 32 * r) : 0u;
-    }
-    // f(r, key) for every position lane + 32 r of this lane, r ascending (uniform trip count)
-    auto for_each_key = [&](auto f) {
-        if (R > 0) {
+            for (int u = 0; u < 8; ++u) {
+                const int i = lane + 32 * (r0 + u);
+                const int ic = min(i, p.P - 1);
+                k[u] = load_key(i);
+                tk[u] = p.tokens[base + ic];
+                tp[u] = __ldcg(p.row_argmax + base + ic);
+            }
 #pragma unroll
-            for (int r = 0; r < kRegs; ++r)
-                if (r < nk) f(r, key_reg[r]);
-        } else {
-            for (int r = 0; r < nk; ++r) f(r, load_key(lane + 32 * r));
+            for (int u = 0; u < 8; ++u) {
+                const int i = lane + 32 * (r0 + u);
+                if (i < kDecideKeys) { stage->key[i] = k[u]; stage->tok[i] = tk[u]; stage->top[i] = tp[u]; }
+            }
         }
-    };
+        __syncwarp();
+    }
+    auto key_at = [&](int r) -> uint32_t { return staged ? stage->key[lane + 32 * r] : load_key(lane + 32 * r); };
     auto score_of = [&](uint32_t key) -> float {     // inverse of the key map (key != 0)
         const float rel = __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
         return kl_mode ? 0.0f - rel : rel;
     };
-    // number of keys of the whole sequence with key >= cand, or key > cand
-    auto count_keys = [&](uint32_t cand, bool strictly) -> int {
-        int cnt = 0;
-        if (R > 0) {
+    // number of keys of the whole sequence with key >= cand, or key > cand.  Staged keys are
+    // also held in registers (up to 32 per lane): the threshold search below makes 33 passes.
+    uint32_t kr[kDecideKeys / 32];
 #pragma unroll
-            for (int r = 0; r < kRegs; ++r) cnt += strictly ? (key_reg[r] > cand) : (key_reg[r] >= cand);
+    for (int r = 0; r < kDecideKeys / 32; ++r) kr[r] = (staged && r < nk) ? stage->key[lane + 32 * r] : 0u;
+    auto count_keys = [&](uint32_t cand, bool strictly) -> int {
+        int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+        if (staged) {
+            const uint32_t bound = strictly ? cand : cand - 1u;      // cand >= 1 when not strict
+#pragma unroll
+            for (int r = 0; r < kDecideKeys / 32; r += 4) {
+                c0 += kr[r] > bound; c1 += kr[r + 1] > bound; c2 += kr[r + 2] > bound; c3 += kr[r + 3] > bound;
+            }
         } else {
-#pragma unroll 8
+#pragma unroll 4
             for (int r = 0; r < nk; ++r) {
                 const uint32_t k = load_key(lane + 32 * r);
-                cnt += strictly ? (k > cand) : (k >= cand);
+                c0 += strictly ? (k > cand) : (k >= cand);
             }
         }
-        return __reduce_add_sync(full, cnt);
+        return __reduce_add_sync(full, c0 + c1 + c2 + c3);
     };
 
     // Eq. 6 normaliser: sum of KL over the drafter-decoded set, in a fixed order
@@ -74,7 +99,10 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
     double kl_sum = 0.0;
     if (kl_mode && p.probabilistic) {
         double part = 0.0;
-        for_each_key([&](int, uint32_t k) { if (k) part += (double)score_of(k); });
+        for (int r = 0; r < nk; ++r) {
+            const uint32_t k = key_at(r);
+            if (k) part += (double)score_of(k);
+        }
         kl_sum = warp_sum(part);
     }
     auto fails = [&](int i, float s) -> bool {
@@ -86,22 +114,20 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
         return u < prob;
     };
 
-    // which of this lane's positions fail (bit r), for up to 32 positions per lane; beyond that
-    // (R == 0 with P > 1024) the rule is evaluated again where it is needed
-    unsigned fail_bits = 0u;
     bool any_fail = false;
-    for_each_key([&](int r, uint32_t k) {
-        const bool f = k != 0u && fails(lane + 32 * r, score_of(k));
-        any_fail |= f;
-        if (r < 32 && f) fail_bits |= 1u << r;
-    });
-    any_fail = __any_sync(full, any_fail);
+    if (p.k > 0 && p.algo != DD_MODE_TRUST) {
+        for (int r = 0; r < nk; ++r) {
+            const uint32_t k = key_at(r);
+            any_fail |= k != 0u && fails(lane + 32 * r, score_of(k));
+        }
+        any_fail = __any_sync(full, any_fail);
+    }
 
     // top-k threshold, needed only if some position fails and fewer than all are protected
     uint32_t thr = 0u;          // k-th largest key
     int quota = 0;              // how many of the positions equal to thr are still kept
     bool topk_active = false, keep_all = false;
-    if (p.k > 0 && any_fail) {
+    if (any_fail) {
         if (n_flagged <= p.k) {
             keep_all = true;
         } else {
@@ -114,45 +140,71 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b)
         }
     }
 
+    // final pass, four positions per lane at a time: first every load of the group (they are
+    // independent, so they overlap), then the decisions and the stores
     int equal_seen = 0;         // positions equal to thr at lower indices
-    for_each_key([&](int r, uint32_t key) {
-        const int i = lane + 32 * r;
-        const long t = base + i;
-        const bool flagged = key != 0u;
-        bool protect = keep_all;
-        if (topk_active) {
-            const bool eq = flagged && key == thr;
-            const unsigned eq_mask = __ballot_sync(full, eq);
-            const int my_rank = equal_seen + __popc(eq_mask & ((1u << lane) - 1u));
-            equal_seen += __popc(eq_mask);
-            protect = key > thr || (eq && my_rank < quota);
+    for (int r0 = 0; r0 < nk; r0 += 4) {
+        uint32_t key[4];
+        int32_t tok[4], top[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = lane + 32 * (r0 + u);
+            const bool in = r0 + u < nk && i < p.P;
+            key[u] = r0 + u < nk ? key_at(r0 + u) : 0u;
+            if (staged) {
+                tok[u] = in ? stage->tok[i] : 0;
+                top[u] = in ? stage->top[i] : 0;
+            } else {
+                tok[u] = in ? p.tokens[base + i] : 0;
+                top[u] = (in && key[u] != 0u) ? __ldcg(p.row_argmax + base + i) : 0;
+            }
         }
-        if (i >= p.P) return;
-        const int32_t tok = p.tokens[t];
-        if (!flagged) {
-            p.out_tokens[t] = tok;
-            p.out_mask[t] = 0;
-            if (p.out_score) p.out_score[t] = 0.0f;
-            return;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int r = r0 + u;
+            if (r >= nk) break;                     // uniform
+            const int i = lane + 32 * r;
+            const long t = base + i;
+            const bool flagged = key[u] != 0u;
+            bool protect = keep_all;
+            if (topk_active) {
+                const bool eq = flagged && key[u] == thr;
+                const unsigned eq_mask = __ballot_sync(full, eq);
+                const int my_rank = equal_seen + __popc(eq_mask & ((1u << lane) - 1u));
+                equal_seen += __popc(eq_mask);
+                protect = key[u] > thr || (eq && my_rank < quota);
+            }
+            if (i >= p.P || dry) continue;
+            if (!flagged) {
+                p.out_tokens[t] = tok[u];
+                p.out_mask[t] = 0;
+                if (p.out_score) p.out_score[t] = 0.0f;
+                continue;
+            }
+            const float s = score_of(key[u]);       // exactly the stored score
+            const bool remask = fails(i, s) && !protect;
+            p.out_mask[t] = remask ? 1 : 0;
+            p.out_tokens[t] = (remask || p.emit_drafter) ? tok[u] : top[u];
+            if (p.out_score) p.out_score[t] = s;
         }
-        const float s = __ldcg(p.row_score + t);
-        const bool failed = r < 32 ? ((fail_bits >> r) & 1u) != 0u : fails(i, s);
-        const bool remask = failed && !protect;
-        p.out_mask[t] = remask ? 1 : 0;
-        p.out_tokens[t] = (remask || p.emit_drafter) ? tok : __ldcg(p.row_argmax + t);
-        if (p.out_score) p.out_score[t] = s;
-    });
+    }
 }
 
-__device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b)
+__device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b, DecideStage *stage)
 {
-    if (p.P <= 256) decide_sequence_impl<8>(p, b);
-    else if (p.P <= 1024) decide_sequence_impl<32>(p, b);
-    else decide_sequence_impl<0>(p, b);
+    decide_sequence_impl(p, b, stage, false);
+}
+
+// Runs the decision code on sequence 0 without storing anything.  The decision runs once per
+// sequence, at the very end of a launch that has streamed the instruction lines out of every
+// cache; a warp with nothing to do yet calls this to bring them back in.
+__device__ __forceinline__ void decide_sequence_rehearsal(const VerifyParams &p, DecideStage *stage)
+{
+    decide_sequence_impl(p, 0, stage, true);
 }
 
 // One sequence has one more completed row; the warp that completes the sequence decides it.
-__device__ __forceinline__ void row_done(const VerifyParams &p, int b)
+__device__ __forceinline__ void row_done(const VerifyParams &p, int b, DecideStage *stage)
 {
     const int lane = threadIdx.x & 31;
     int last = 0;
@@ -164,21 +216,28 @@ __device__ __forceinline__ void row_done(const VerifyParams &p, int b)
     if (!last) return;
     __threadfence();
     if (lane == 0) p.seq_counter[b] = 0u;      // ready for the next launch
-    decide_sequence(p, b);
+    decide_sequence(p, b, stage);
 }
 
-// The calling warp saw the row's last chunk published: fold the row's partials in chunk
-// order (fp64), store the row's score and argmax, and report the row to its sequence.
+// 16 bytes from shared or global memory, never from a stale cache line or register copy.
+__device__ __forceinline__ float4 ld_volatile16(const void *ptr)
+{
+    float4 r;
+    asm volatile("ld.volatile.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(ptr));
+    return r;
+}
+
+// Folds n chunk partials of one row, in chunk order, in fp64 (warp-level; src may point to
+// shared or global memory).  Every lane returns the row's score (KL_i of Eq. 5, or c_i of
+// Eq. 7) and the lowest index of the verifier's maximum.
 template <bool KL>
-__device__ __forceinline__ void fold_row(const VerifyParams &p, int row)
+__device__ __noinline__ void fold_partials(const Partial *src, int n, float &score, int &argmax)
 {
     const int lane = threadIdx.x & 31;
-    __threadfence();
-    const Partial *src = p.partials + (size_t)row * p.nchunks;
     float bm_v = -INFINITY, bm_d = -INFINITY;
     int bidx = 0x7FFFFFFF;
-    for (int ch = lane; ch < p.nchunks; ch += 32) {
-        const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + ch));
+    for (int ch = lane; ch < n; ch += 32) {
+        const float4 a = ld_volatile16(src + ch);
         const float mv = a.x, md = a.w;
         const int ix = __float_as_int(a.z);
         if (mv > bm_v || (mv == bm_v && ix < bidx)) { bm_v = mv; bidx = ix; }
@@ -193,9 +252,9 @@ __device__ __forceinline__ void fold_row(const VerifyParams &p, int row)
     }
     const float Mv = bm_v * kLog2e, Md = bm_d * kLog2e;
     double sv = 0.0, sd = 0.0, tt = 0.0;
-    for (int ch = lane; ch < p.nchunks; ch += 32) {
-        const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + ch));
-        const float4 bq = __ldcg(reinterpret_cast<const float4 *>(src + ch) + 1);
+    for (int ch = lane; ch < n; ch += 32) {
+        const float4 a = ld_volatile16(src + ch);
+        const float4 bq = ld_volatile16(reinterpret_cast<const float4 *>(src + ch) + 1);
         sv += (double)a.y * exp2((double)(a.x * kLog2e) - (double)Mv);
         if (KL) {
             const double f = exp2((double)(a.w * kLog2e) - (double)Md);
@@ -205,23 +264,39 @@ __device__ __forceinline__ void fold_row(const VerifyParams &p, int row)
     }
     sv = warp_sum(sv);
     if (KL) { sd = warp_sum(sd); tt = warp_sum(tt); }
+    float sc = 0.f;
     if (lane == 0) {
-        float score;
         if (KL) {
             const double lse_v = (double)Mv * kLn2 + log(sv);
             const double lse_d = (double)Md * kLn2 + log(sd);
             const double kl = tt / sd - lse_d + lse_v;
-            score = (float)fmax(kl, 0.0);
+            sc = (float)fmax(kl, 0.0);
         } else {
             // the maximum's own term is 2^(m*log2e - M), not exactly 1
-            score = (float)(exp2((double)bm_v * (double)kLog2e - (double)Mv) / sv);
+            sc = (float)(exp2((double)bm_v * (double)kLog2e - (double)Mv) / sv);
         }
+    }
+    score = __shfl_sync(0xFFFFFFFFu, sc, 0);
+    argmax = bidx;
+}
+
+// The calling warp saw the row's last chunk published to global memory: fold the row, store
+// its score and argmax, and report the row to its sequence.
+template <bool KL>
+__device__ __forceinline__ void fold_row(const VerifyParams &p, int row, DecideStage *stage)
+{
+    const int lane = threadIdx.x & 31;
+    __threadfence();
+    float score;
+    int argmax;
+    fold_partials<KL>(p.partials + (size_t)row * p.nchunks, p.nchunks, score, argmax);
+    if (lane == 0) {
         __stcg(p.row_score + row, score);
-        __stcg(p.row_argmax + row, bidx);
+        __stcg(p.row_argmax + row, argmax);
         p.row_counter[row] = 0u;      // ready for the next launch
     }
     __syncwarp();
-    row_done(p, row / p.P);
+    row_done(p, row / p.P, stage);
 }
 
 // Publishes up to 32 finished (row, chunk) partials at once -- lane l holds entry l, its row in
@@ -229,7 +304,7 @@ __device__ __forceinline__ void fold_row(const VerifyParams &p, int row)
 // whose last chunk was among them are then folded one after the other.  An entry with a
 // negative chunk stands for an unflagged row, which is only reported to its sequence.
 template <bool KL>
-__device__ __forceinline__ void publish_batch(const VerifyParams &p, const Partial &c, int n)
+__device__ __forceinline__ void publish_batch(const VerifyParams &p, const Partial &c, int n, DecideStage *stage)
 {
     const int lane = threadIdx.x & 31;
     const unsigned full = 0xFFFFFFFFu;
@@ -249,23 +324,23 @@ __device__ __forceinline__ void publish_batch(const VerifyParams &p, const Parti
     while (todo) {
         const int src = __ffs(todo) - 1;
         todo &= todo - 1;
-        fold_row<KL>(p, __shfl_sync(full, row, src));
+        fold_row<KL>(p, __shfl_sync(full, row, src), stage);
     }
     todo = __ballot_sync(full, mine && chunk < 0);
     while (todo) {
         const int src = __ffs(todo) - 1;
         todo &= todo - 1;
-        row_done(p, __shfl_sync(full, row, src) / p.P);
+        row_done(p, __shfl_sync(full, row, src) / p.P, stage);
     }
 }
 
 // One partial, held by every lane alike.
 template <bool KL>
-__device__ __forceinline__ void chunk_done(const VerifyParams &p, int row, int chunk, Partial c)
+__device__ __forceinline__ void chunk_done(const VerifyParams &p, int row, int chunk, Partial c, DecideStage *stage)
 {
     c.pad0 = __int_as_float(row);
     c.pad1 = __int_as_float(chunk);
-    publish_batch<KL>(p, c, 1);
+    publish_batch<KL>(p, c, 1, stage);
 }
 
 }  // namespace ddv

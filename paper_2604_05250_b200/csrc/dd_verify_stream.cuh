@@ -1,16 +1,20 @@
 // Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
 //
-// One persistent CTA per SM: fifteen warps stream, one warp publishes.  A streaming
-// warp takes a (row, chunk) of 4096 logits from the CTA's queue and pulls it through
-// its private ring of three shared-memory stages in pieces of 1024 logits per tensor
-// with bulk asynchronous copies (cp.async.bulk + mbarrier), so loads stay in flight
-// while the warp computes.  Within a chunk every lane keeps its own running maxima,
-// reference points and sums (packed bf16x2 maxima, packed fp32 pairs); lanes talk to
-// each other only when the chunk ends.  The finished partial goes into a
-// shared-memory queue; the publishing warp drains it in batches (one fence per batch),
-// counts chunks per row, folds completed rows and decides completed sequences, so the
-// streaming warps never wait for a round trip to global memory.  No CTA-wide barrier
-// follows start-up.
+// One persistent CTA per SM: fifteen warps stream, one warp publishes.  The flagged rows'
+// (row, chunk) units, 4096 logits each, are numbered in row order and cut into equal
+// contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  A
+// streaming warp takes the next unit of the range and pulls it through its private ring
+// of shared-memory stages in pieces of 1024 logits per tensor with bulk asynchronous
+// copies (cp.async.bulk + mbarrier), so loads stay in flight while the warp computes.
+// Within a chunk every lane keeps its own running maxima, reference points and sums
+// (packed bf16x2 maxima, packed fp32 pairs); lanes talk to each other only when the
+// chunk ends.  The chunk's partial goes into a table in shared memory; the warp that
+// stores a row's last chunk folds the row there, so a row that lies inside one range
+// costs no global round trip.  Rows cut by a range boundary go through global memory as
+// chunk partials plus one counter update per range.  The publishing warp takes finished
+// rows from a shared-memory queue, stores their scores, updates the sequence counters in
+// batches (one fence per batch) and decides completed sequences, so the streaming warps
+// never wait for global memory.
 #pragma once
 
 #include "dd_verify_common.cuh"
@@ -24,7 +28,8 @@ constexpr int kSQueue = 64;                                   // finished-chunk 
 constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits: one ring stage per tensor
 constexpr int kPiecesPerChunk = 4;
 constexpr int kSChunk = kPiece * kPiecesPerChunk;             // 4096 logits per (row, chunk)
-constexpr int kSStages = 3;
+constexpr int kSStages = 2;
+constexpr int kSTable = 768;                                  // chunk partials a CTA keeps per range
 constexpr unsigned kErrWaitPiece = 0x700, kErrWaitQueue = 0x800;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *ptr)
@@ -63,33 +68,10 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return r;
 }
 
-// Packed fp32 pairs (one instruction works on two values).
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c)
-{
-    unsigned long long r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b)
-{
-    unsigned long long r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
 struct PieceDesc {     // what a ring stage holds; row < 0: nothing more will come
     int row, chunk, e_begin, n;
-    int ordinal, last, pad0, pad1;   // ordinal: piece number within its chunk
+    int ordinal, last;     // ordinal: piece number within its chunk
+    int slot, local_row;   // the chunk's slot in the CTA's table, its row's number within the range
 };
 
 // Running state of one lane over the pieces of a chunk.
@@ -97,7 +79,7 @@ struct LaneState {
     uint32_t max2_v, max2_d;   // packed bf16x2 running maxima (even / odd logits of the lane's words)
     uint32_t where2_v;         // per half: ordinal of the word that first attained the verifier's maximum
     float M_v, M_d;            // reference points: lane maximum * log2e
-    unsigned long long s_v, s_d, t;   // packed fp32 pairs (even / odd logits)
+    float2 s_v, s_d, t;        // sums of the even / odd logits
 };
 
 __device__ __forceinline__ void lane_reset(LaneState &L)
@@ -105,11 +87,12 @@ __device__ __forceinline__ void lane_reset(LaneState &L)
     L.max2_v = L.max2_d = 0xFF80FF80u;     // -inf, -inf
     L.where2_v = 0u;
     L.M_v = L.M_d = -INFINITY;
-    L.s_v = L.s_d = L.t = 0ull;
+    L.s_v = L.s_d = L.t = make_float2(0.f, 0.f);
 }
 
 // One piece (n logits, a multiple of 8; lane's vector j covers logits (lane + 32 j) * 8 ..+7).
-template <bool KL>
+// kFull: n == kPiece, no vector is absent.
+template <bool KL, bool kFull>
 __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecPerThread],
                                            const uint4 (&rd)[kVecPerThread], int n, int lane, int ordinal)
 {
@@ -149,41 +132,38 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
     const float M_v = fmaxf(bf16lo(max2_v), bf16hi(max2_v)) * kLog2e;
     {
         const float f = rescale_factor(L.M_v, M_v);
-        L.s_v = fma2(L.s_v, pack2(f, f), 0ull);
+        L.s_v = __fmul2_rn(L.s_v, make_float2(f, f));
         L.M_v = M_v;
     }
     float M_d = 0.f;
     if (KL) {
         M_d = fmaxf(bf16lo(max2_d), bf16hi(max2_d)) * kLog2e;
         const float f = rescale_factor(L.M_d, M_d);
-        const unsigned long long f2 = pack2(f, f);
-        L.s_d = fma2(L.s_d, f2, 0ull);
-        L.t = fma2(L.t, f2, 0ull);
+        L.s_d = __fmul2_rn(L.s_d, make_float2(f, f));
+        L.t = __fmul2_rn(L.t, make_float2(f, f));
         L.M_d = M_d;
     }
     // pass 2: one ex2 per logit against the lane's reference
-    const unsigned long long log2e2 = pack2(kLog2e, kLog2e);
-    const unsigned long long nMv2 = pack2(-M_v, -M_v), nMd2 = pack2(-M_d, -M_d);
-    const unsigned long long neg1 = pack2(-1.f, -1.f);
-    unsigned long long s_v = L.s_v, s_d = L.s_d, t = L.t;
+    const float2 log2e2 = make_float2(kLog2e, kLog2e);
+    const float2 nMv2 = make_float2(-M_v, -M_v), nMd2 = make_float2(-M_d, -M_d);
+    const float2 neg1 = make_float2(-1.f, -1.f);
+    float2 s_v = L.s_v, s_d = L.s_d, t = L.t;
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
-        if ((lane + j * 32) * 8 < n) {
+        if (kFull || (lane + j * 32) * 8 < n) {
             const uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
             const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const unsigned long long v2 = pack2(bf16lo(wv[h]), bf16hi(wv[h]));
-                float a0, a1;
-                unpack2(fma2(v2, log2e2, nMv2), a0, a1);
-                s_v = add2(s_v, pack2(ex2_approx(a0), ex2_approx(a1)));
+                const float2 v2 = make_float2(bf16lo(wv[h]), bf16hi(wv[h]));
+                const float2 a = __ffma2_rn(v2, log2e2, nMv2);
+                s_v = __fadd2_rn(s_v, make_float2(ex2_approx(a.x), ex2_approx(a.y)));
                 if (KL) {
-                    const unsigned long long d2 = pack2(bf16lo(wd[h]), bf16hi(wd[h]));
-                    float b0, b1;
-                    unpack2(fma2(d2, log2e2, nMd2), b0, b1);
-                    const unsigned long long e2 = pack2(ex2_approx(b0), ex2_approx(b1));
-                    s_d = add2(s_d, e2);
-                    t = fma2(e2, fma2(v2, neg1, d2), t);          // e * (d - v)
+                    const float2 d2 = make_float2(bf16lo(wd[h]), bf16hi(wd[h]));
+                    const float2 b = __ffma2_rn(d2, log2e2, nMd2);
+                    const float2 e2 = make_float2(ex2_approx(b.x), ex2_approx(b.y));
+                    s_d = __fadd2_rn(s_d, e2);
+                    t = __ffma2_rn(e2, __ffma2_rn(v2, neg1, d2), t);          // e * (d - v)
                 }
             }
         }
@@ -205,16 +185,12 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
     const int e_lo = element_of(L.where2_v & 0xFFFFu, 0), e_hi = element_of(L.where2_v >> 16, 1);
     c.m_v = fmaxf(lo_m, hi_m);
     c.idx = lo_m > hi_m ? e_lo : (hi_m > lo_m ? e_hi : min(e_lo, e_hi));
-    float a0, a1;
-    unpack2(L.s_v, a0, a1);
-    c.s_v = a0 + a1;
+    c.s_v = L.s_v.x + L.s_v.y;
     c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f;
     if (KL) {
         c.m_d = fmaxf(bf16lo(L.max2_d), bf16hi(L.max2_d));
-        unpack2(L.s_d, a0, a1);
-        c.s_d = a0 + a1;
-        unpack2(L.t, a0, a1);
-        c.t = a0 + a1;
+        c.s_d = L.s_d.x + L.s_d.y;
+        c.t = L.t.x + L.t.y;
     }
     c.pad0 = c.pad1 = 0.f;
 #pragma unroll
@@ -241,19 +217,32 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
     return c;
 }
 
-// Queue of finished chunks between the streaming warps (many producers) and the publishing
-// warp (one consumer), in shared memory.
-struct ChunkQueue {
-    Partial entry[kSQueue];
+// A finished row (or a range's share of a row cut by a range boundary), handed from a
+// streaming warp to the publishing warp.
+struct RowEvent {
+    int row;
+    int whole;        // 1: the row lay inside the range and is folded: score and argmax are final
+    float score;
+    int argmax;
+    int first_slot;   // whole == 0: the range's chunks of this row are table slots first_slot ..
+    int first_chunk;  //             and chunks first_chunk .. of the row,
+    int count;        //             count of them
+    int pad;
+};
+
+// Queue of row events between the streaming warps (many producers) and the publishing warp
+// (one consumer), in shared memory.
+struct EventQueue {
+    RowEvent entry[kSQueue];
     unsigned int ready[kSQueue];     // sequence number + 1 of the entry the slot holds
     unsigned int tail;               // next sequence number to hand out
     unsigned int head;               // entries below this have been taken
-    unsigned int done;               // streaming warps that have finished
+    unsigned int done;               // streaming warps that have finished the current range
     unsigned int pad;
 };
 
 // One lane of a streaming warp hands over an entry.  False if the queue stayed full.
-__device__ __forceinline__ bool queue_push(ChunkQueue &q, const Partial &e)
+__device__ __forceinline__ bool queue_push(EventQueue &q, const RowEvent &e)
 {
     const unsigned int seq = atomicAdd(&q.tail, 1u);
     volatile unsigned int *head = &q.head;
