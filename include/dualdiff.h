@@ -131,9 +131,9 @@ int dd_verify_host(const void *drafter_logits, const void *verifier_logits,
  * cudaMalloc/cudaFree, or that does not own the allocator of its process: this
  * call performs no cudaMalloc, cudaFree or other allocating routine.  Its scratch
  * (chunk partials, row results, completion counters) is a fixed array of about
- * 4.3 MB inside the library, held by every GPU that loads the library until the
+ * 2.1 MB inside the library, held by every GPU that loads the library until the
  * process exits.
- * Limits: B*P <= 4096 and B*P*ceil(V/4096) <= 131072; larger problems return
+ * Limits: B*P <= 4096 and B*P*ceil(V/8192) <= 65536; larger problems return
  * DD_ERR_UNSUPPORTED and launch nothing.
  * The first call on each device looks up the array's device address; make that
  * first call outside any stream capture.  All calls on a device share the one

@@ -10,8 +10,8 @@
 // each logit is read from HBM exactly once.
 //
 // Streaming kernel (V % 8 == 0, 16-byte aligned logits; dd_verify_stream.cuh):
-// persistent CTAs whose warps stream chunks of 4096 logits through private
-// shared-memory rings fed by bulk asynchronous copies.
+// persistent CTAs whose warps stream chunks of 8192 logits with the next piece's
+// loads in flight while the current one is computed.
 // Element-wise kernel (any V, any alignment; this file): one CTA of 256 threads
 // per chunk of at most 8192 logits, 2-byte loads with bounds checks.
 //
@@ -219,18 +219,16 @@ int launch_stream(const VerifyParams &p, cudaStream_t stream)
 {
     static bool attr_done[64] = {};
     static int sm_count[64] = {};
-    constexpr int smem = kSStreamWarps * kSStages * (KL ? 2 : 1) * kPiece * 2;
     int dev = 0;
     DD_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return dd::cuda_fail(cudaErrorInvalidDevice, "dd_verify: device index");
     if (!attr_done[dev]) {
-        DD_CUDA_TRY(cudaFuncSetAttribute(verify_stream_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         DD_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
         attr_done[dev] = true;
     }
     const long units = (long)p.B * p.P * p.nchunks;
     const long grid = units < sm_count[dev] ? units : sm_count[dev];
-    verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, smem, stream>>>(p);
+    verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, 0, stream>>>(p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
     return DD_OK;
@@ -369,7 +367,7 @@ extern "C" int dd_verify_status(void)
 namespace {
 
 constexpr int kStaticMaxRows = 4096;          // B * P
-constexpr int kStaticMaxPartials = 131072;    // B * P * ceil(V / 4096)
+constexpr int kStaticMaxPartials = 65536;     // B * P * ceil(V / 8192)
 constexpr size_t kStaticCounterBytes = (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255)) +
                                        (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));   // rows + sequences
 constexpr size_t kStaticRowBytes = 2 * (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));  // score + argmax

@@ -1,20 +1,22 @@
 // Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
 //
 // One persistent CTA per SM: fifteen warps stream, one warp publishes.  The flagged rows'
-// (row, chunk) units, 4096 logits each, are numbered in row order and cut into equal
-// contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  A
-// streaming warp takes the next unit of the range and pulls it through its private ring
-// of shared-memory stages in pieces of 1024 logits per tensor with bulk asynchronous
-// copies (cp.async.bulk + mbarrier), so loads stay in flight while the warp computes.
-// Within a chunk every lane keeps its own running maxima, reference points and sums
-// (packed bf16x2 maxima, packed fp32 pairs); lanes talk to each other only when the
-// chunk ends.  The chunk's partial goes into a table in shared memory; the warp that
-// stores a row's last chunk folds the row there, so a row that lies inside one range
-// costs no global round trip.  Rows cut by a range boundary go through global memory as
-// chunk partials plus one counter update per range.  The publishing warp takes finished
-// rows from a shared-memory queue, stores their scores, updates the sequence counters in
-// batches (one fence per batch) and decides completed sequences, so the streaming warps
-// never wait for global memory.
+// (row, chunk) units, 8192 logits each, are numbered in row order and cut into equal
+// contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  The
+// range's units go to the streaming warps in turn.  A warp walks its unit in pieces of 1024
+// logits per tensor: every lane holds four 16-byte vectors per tensor of the current piece
+// in registers and has the loads of the next piece in flight while it computes (the
+// measured copy bandwidth is reached with this depth; a shared-memory ring fed by bulk
+// copies reached it too but cost about four times the instructions per piece).  Within a
+// chunk every lane keeps its own running maxima, reference points and sums (packed bf16x2
+// maxima, packed fp32 pairs); lanes talk to each other only when the chunk ends.  The
+// chunk's partial goes into a table in shared memory; the warp that stores a row's last
+// chunk folds the row there, so a row that lies inside one range costs no global round
+// trip.  Rows cut by a range boundary go through global memory as chunk partials plus one
+// counter update per range.  The publishing warp takes finished rows from a shared-memory
+// queue, stores their scores, updates the sequence counters in batches (one fence per
+// batch) and decides completed sequences, so the streaming warps never wait for global
+// memory other than their logits.
 #pragma once
 
 #include "dd_verify_common.cuh"
@@ -25,54 +27,19 @@ constexpr int kSStreamWarps = 15;                             // warps that stre
 constexpr int kSWarps = kSStreamWarps + 1;                    // + one that publishes finished chunks
 constexpr int kSThreads = kSWarps * 32;
 constexpr int kSQueue = 64;                                   // finished-chunk queue slots
-constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits: one ring stage per tensor
-constexpr int kPiecesPerChunk = 4;
-constexpr int kSChunk = kPiece * kPiecesPerChunk;             // 4096 logits per (row, chunk)
-constexpr int kSStages = 2;
+constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per step of a warp
+constexpr int kPiecesPerChunk = 8;
+constexpr int kSChunk = kPiece * kPiecesPerChunk;             // 8192 logits per (row, chunk)
 constexpr int kSTable = 768;                                  // chunk partials a CTA keeps per range
-constexpr unsigned kErrWaitPiece = 0x700, kErrWaitQueue = 0x800;
+constexpr unsigned kErrWaitQueue = 0x800;
 
-__device__ __forceinline__ uint32_t smem_u32(const void *ptr)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Untiled bulk copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr)
+__device__ __forceinline__ uint4 ld_stream(const uint4 *ptr)
 {
     uint4 r;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(ptr));
     return r;
 }
-
-struct PieceDesc {     // what a ring stage holds; row < 0: nothing more will come
-    int row, chunk, e_begin, n;
-    int ordinal, last;     // ordinal: piece number within its chunk
-    int slot, local_row;   // the chunk's slot in the CTA's table, its row's number within the range
-};
 
 // Running state of one lane over the pieces of a chunk.
 struct LaneState {
@@ -171,11 +138,11 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
     L.s_v = s_v; L.s_d = s_d; L.t = t;
 }
 
-// The chunk has ended: the 32 lane states become one partial (lane 0's copy is the one used).
+// The chunk has ended: the 32 lane states become one partial (the same bits in every lane):
+// the warp's maxima first, then every lane's sums moved to them and added up.
 template <bool KL>
 __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chunk_begin, int lane)
 {
-    const unsigned full = 0xFFFFFFFFu;
     Partial c;
     const float lo_m = bf16lo(L.max2_v), hi_m = bf16hi(L.max2_v);
     auto element_of = [&](uint32_t q, int odd) {     // q = piece * 16 + j * 4 + h
@@ -183,37 +150,22 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
                2 * (int)(q & 3u) + odd;
     };
     const int e_lo = element_of(L.where2_v & 0xFFFFu, 0), e_hi = element_of(L.where2_v >> 16, 1);
-    c.m_v = fmaxf(lo_m, hi_m);
-    c.idx = lo_m > hi_m ? e_lo : (hi_m > lo_m ? e_hi : min(e_lo, e_hi));
-    c.s_v = L.s_v.x + L.s_v.y;
+    const float my_m = fmaxf(lo_m, hi_m);
+    const int my_idx = lo_m > hi_m ? e_lo : (hi_m > lo_m ? e_hi : min(e_lo, e_hi));
+    c.m_v = warp_max(my_m);
+    int idx = my_m == c.m_v ? my_idx : 0x7FFFFFFF;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) idx = min(idx, __shfl_xor_sync(0xFFFFFFFFu, idx, o));
+    c.idx = idx;
+    c.s_v = warp_sum((L.s_v.x + L.s_v.y) * rescale_factor(L.M_v, c.m_v * kLog2e));
     c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f;
     if (KL) {
-        c.m_d = fmaxf(bf16lo(L.max2_d), bf16hi(L.max2_d));
-        c.s_d = L.s_d.x + L.s_d.y;
-        c.t = L.t.x + L.t.y;
+        c.m_d = warp_max(fmaxf(bf16lo(L.max2_d), bf16hi(L.max2_d)));
+        const float f = rescale_factor(L.M_d, c.m_d * kLog2e);
+        c.s_d = warp_sum((L.s_d.x + L.s_d.y) * f);
+        c.t = warp_sum((L.t.x + L.t.y) * f);
     }
     c.pad0 = c.pad1 = 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        Partial other;
-        other.m_v = __shfl_xor_sync(full, c.m_v, o);
-        other.s_v = __shfl_xor_sync(full, c.s_v, o);
-        other.idx = __shfl_xor_sync(full, c.idx, o);
-        other.m_d = 0.f; other.s_d = 0.f; other.t = 0.f;
-        if (KL) {
-            other.m_d = __shfl_xor_sync(full, c.m_d, o);
-            other.s_d = __shfl_xor_sync(full, c.s_d, o);
-            other.t = __shfl_xor_sync(full, c.t, o);
-        }
-        // both lanes of a pair merge (lower lane's, upper lane's) in that order: same bits in both
-        if ((lane & o) == 0) {
-            merge_partial<KL>(c, other);
-        } else {
-            merge_partial<KL>(other, c);
-            c.m_v = other.m_v; c.s_v = other.s_v; c.idx = other.idx;
-            c.m_d = other.m_d; c.s_d = other.s_d; c.t = other.t;
-        }
-    }
     return c;
 }
 

@@ -40,27 +40,16 @@ __device__ __forceinline__ void rows_done(const VerifyParams &p, SeqTally &tally
 template <bool KL>
 __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const VerifyParams p)
 {
-    extern __shared__ __align__(128) unsigned char ring_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[kSStreamWarps][kSStages];
-    __shared__ __align__(16) PieceDesc s_desc[kSStreamWarps][kSStages];
     __shared__ __align__(16) Partial s_table[kSTable];          // chunk partials of the current range
     __shared__ int s_rows[kSTable + 2];                          // flagged rows the range touches
     __shared__ unsigned int s_rowcnt[kSTable + 2];               // their chunks stored so far
     __shared__ __align__(16) EventQueue s_queue;
-    __shared__ unsigned int s_next;
     __shared__ int s_scan[kSWarps];
     __shared__ DecideStage s_decide;                              // decision stage (publishing warp only)
 
-    constexpr int kTensorBytes = kPiece * 2;                      // one piece of one tensor
-    constexpr int kStageBytes = (KL ? 2 : 1) * kTensorBytes;
     const unsigned full = 0xFFFFFFFFu;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nch = p.nchunks;
-
-    if (warp < kSStreamWarps && lane == 0) {
-        for (int s = 0; s < kSStages; ++s) mbar_init(smem_u32(&s_bar[warp][s]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
 
     // ---- every thread counts the flagged rows of its contiguous slice of the B*P rows; the block
     // scan gives each thread the number of flagged rows before its slice, and the total
@@ -105,8 +94,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     }
 
     bool rehearsed = false;
-    unsigned ring_uses = 0;       // streaming warps: pieces taken from the ring so far
-    bool wait_ok = true, queue_ok = true;
+    bool queue_ok = true;
 
     for (long range = blockIdx.x; range < n_ranges; range += gridDim.x) {
         const long lo = total_units * range / n_ranges, hi = total_units * (range + 1) / n_ranges;
@@ -126,7 +114,6 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             for (int i = tid; i < (int)(f_hi - f_lo + 1); i += kSThreads) s_rowcnt[i] = 0u;
             if (tid < kSQueue) s_queue.ready[tid] = 0u;
             if (tid == 0) {
-                s_next = 0u;
                 s_queue.tail = s_queue.head = s_queue.done = 0u;
             }
         }
@@ -166,7 +153,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                         if (lane == 0 && p.status) atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
                         break;
                     }
-                    __nanosleep(100);
+                    __nanosleep(250);
                     continue;
                 }
                 idle = 0;
@@ -228,120 +215,117 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         }
 
         // =================================================================== streaming warps
-        const uint32_t ring = smem_u32(ring_raw) + warp * (kSStages * kStageBytes);
-        const uint32_t bars = smem_u32(&s_bar[warp][0]);
+        const unsigned ulo = (unsigned)lo, uhi = (unsigned)hi, uflo = (unsigned)f_lo;   // units fit 31 bits
+        const int last_pieces = (p.V - (nch - 1) * kSChunk + kPiece - 1) / kPiece;       // of a row's last chunk
 
-        // ---- producer side (all lanes follow, lane 0 issues): the unit being fed into the ring
-        int pu_row = 0, pu_chunk = 0, pu_e = 0, pu_begin = 0, pu_end = 0, pu_slot = 0, pu_local = 0;
-        bool pu_done = !wait_ok;          // after an expired wait this warp only reports itself done
-        auto produce = [&](int stage) {
-            for (;;) {
-                if (pu_done) {
-                    if (lane == 0) s_desc[warp][stage].row = -1;
-                    return;
+        // Units of the range go to the streaming warps in turn: warp w takes units w, w + 15, ...
+        // A cursor walks one warp's pieces in order (all lanes hold the same values).
+        struct Cursor {
+            int t;              // unit within the range (= its table slot); >= n_units: past the end
+            int local_row;      // the unit's row, numbered within the range
+            int chunk, piece, npieces, row;
+        };
+        auto enter_unit = [&](Cursor &c) {
+            if (c.t >= n_units) return;
+            c.npieces = c.chunk == nch - 1 ? last_pieces : kPiecesPerChunk;
+            c.row = s_rows[c.local_row];
+        };
+        auto advance = [&](Cursor &c) {
+            if (++c.piece < c.npieces) return;
+            c.piece = 0;
+            c.t += kSStreamWarps;
+            c.chunk += kSStreamWarps;
+            if (c.chunk >= nch) {
+                const int q = c.chunk / nch;
+                c.chunk -= q * nch;
+                c.local_row += q;
+            }
+            enter_unit(c);
+        };
+        // the lane's vectors of the cursor's piece: four per tensor, -inf where the row has ended
+        auto fetch = [&](const Cursor &c, uint4 (&v)[kVecPerThread], uint4 (&d)[kVecPerThread]) {
+            const int e_begin = c.chunk * kSChunk + c.piece * kPiece;
+            const int n = p.V - e_begin;                      // logits left in the row
+            const size_t off = (size_t)c.row * p.V + e_begin;
+            const uint4 *gv = reinterpret_cast<const uint4 *>(p.verifier + off) + lane;
+            const uint4 *gd = reinterpret_cast<const uint4 *>(p.drafter + off) + lane;
+            if (n >= kPiece) {
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    v[j] = ld_stream(gv + 32 * j);
+                    if (KL) d[j] = ld_stream(gd + 32 * j);
                 }
-                if (pu_e < pu_end) {
-                    const int n = min(kPiece, pu_end - pu_e);
-                    if (lane == 0) {
-                        PieceDesc d;
-                        d.row = pu_row; d.chunk = pu_chunk; d.e_begin = pu_e; d.n = n;
-                        d.ordinal = (pu_e - pu_begin) / kPiece; d.last = pu_e + n >= pu_end;
-                        d.slot = pu_slot; d.local_row = pu_local;
-                        s_desc[warp][stage] = d;
-                        const uint32_t bytes = (uint32_t)n * 2u;
-                        const uint32_t bar = bars + 8 * stage, dst = ring + stage * kStageBytes;
-                        const size_t off = (size_t)pu_row * p.V + pu_e;
-                        mbar_expect_tx(bar, KL ? 2 * bytes : bytes);
-                        bulk_load(dst, p.verifier + off, bytes, bar);
-                        if (KL) bulk_load(dst + kTensorBytes, p.drafter + off, bytes, bar);
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    const bool in = (lane + 32 * j) * 8 < n;
+                    v[j] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+                    if (KL) d[j] = v[j];
+                    if (in) {
+                        v[j] = ld_stream(gv + 32 * j);
+                        if (KL) d[j] = ld_stream(gd + 32 * j);
                     }
-                    pu_e += n;
-                    return;
                 }
-                // next unit of the range
-                unsigned int t = 0;
-                if (lane == 0) t = atomicAdd(&s_next, 1u);
-                t = __shfl_sync(full, t, 0);
-                if (t >= (unsigned)n_units) { pu_done = true; continue; }
-                const long unit = lo + t;
-                const long f = unit / nch;
-                pu_chunk = (int)(unit - f * nch);
-                pu_local = (int)(f - f_lo);
-                pu_row = s_rows[pu_local];
-                pu_slot = (int)t;
-                pu_begin = pu_e = pu_chunk * kSChunk;
-                pu_end = min(p.V, pu_begin + kSChunk);
+            }
+            if (!KL) {
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) d[j] = make_uint4(0u, 0u, 0u, 0u);
             }
         };
 
-        // the ring is empty here; its stages continue in order across ranges
-        for (int s = 0; s < kSStages; ++s) produce((ring_uses + s) % kSStages);
-        __syncwarp();
+        Cursor cc;
+        {
+            cc.t = warp;
+            cc.piece = 0; cc.npieces = 0; cc.row = 0;
+            const unsigned unit = ulo + (unsigned)warp, f = unit / (unsigned)nch;
+            cc.chunk = (int)(unit - f * (unsigned)nch);
+            cc.local_row = (int)(f - uflo);
+            enter_unit(cc);
+        }
+        Cursor nc = cc;                                       // the piece whose loads are in flight
+        uint4 nv[kVecPerThread], nd[kVecPerThread];
+        if (nc.t < n_units) fetch(nc, nv, nd);
 
         LaneState L;
         lane_reset(L);
-        for (;; ++ring_uses) {
-            const int stage = ring_uses % kSStages;
-            const uint32_t parity = (ring_uses / kSStages) & 1u;
-            const PieceDesc d = s_desc[warp][stage];
-            if (d.row < 0) break;
-
-            // bounded, warp-uniform wait for the stage's copies
-            bool landed = false;
-            for (unsigned it = 0; it < (1u << 22); ++it) {
-                landed = mbar_try_wait(bars + 8 * stage, parity);
-                if (__all_sync(full, landed)) { landed = true; break; }
-                landed = false;
-                if (it > 64) __nanosleep(32);
-            }
-            if (!landed) { wait_ok = false; break; }
-
+        while (cc.t < n_units) {
             uint4 rv[kVecPerThread], rd[kVecPerThread];
-            const uint32_t src = ring + stage * kStageBytes;
-            const bool whole_piece = d.n == kPiece;
 #pragma unroll
-            for (int j = 0; j < kVecPerThread; ++j) {
-                const int e0 = (lane + j * 32) * 8;
-                if (whole_piece || e0 < d.n) {
-                    rv[j] = lds128(src + e0 * 2);
-                    if (KL) rd[j] = lds128(src + kTensorBytes + e0 * 2);
-                    else rd[j] = make_uint4(0u, 0u, 0u, 0u);
-                } else {
-                    rv[j] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-                    rd[j] = rv[j];
-                }
-            }
-            __syncwarp();          // every lane has its vectors: the stage can be refilled
-            produce(stage);
-            __syncwarp();
+            for (int j = 0; j < kVecPerThread; ++j) { rv[j] = nv[j]; rd[j] = nd[j]; }
+            advance(nc);
+            if (nc.t < n_units) fetch(nc, nv, nd);            // in flight while this piece is computed
 
-            if (whole_piece) lane_piece<KL, true>(L, rv, rd, d.n, lane, d.ordinal);
-            else lane_piece<KL, false>(L, rv, rd, d.n, lane, d.ordinal);
-            if (!d.last) continue;
+            const int n = min(kPiece, p.V - (cc.chunk * kSChunk + cc.piece * kPiece));
+            if (n == kPiece) lane_piece<KL, true>(L, rv, rd, n, lane, cc.piece);
+            else lane_piece<KL, false>(L, rv, rd, n, lane, cc.piece);
+            const bool chunk_ends = cc.piece == cc.npieces - 1;
+            const Cursor done = cc;
+            advance(cc);
+            if (!chunk_ends) continue;
 
             // ---- the chunk is complete: into the table; the warp that completes the range's share
             // of a row hands the row on
-            const Partial part = lanes_to_partial<KL>(L, d.chunk * kSChunk, lane);
+            const Partial part = lanes_to_partial<KL>(L, done.chunk * kSChunk, lane);
             lane_reset(L);
-            const long f = f_lo + d.local_row;
-            const long first_unit = max(lo, f * nch), end_unit = min(hi, (f + 1) * nch);
+            const unsigned row_first = (uflo + (unsigned)done.local_row) * (unsigned)nch;   // the row's unit 0
+            const unsigned first_unit = max(ulo, row_first), end_unit = min(uhi, row_first + (unsigned)nch);
             const int share = (int)(end_unit - first_unit);
             int complete = 0;
             if (lane == 0) {
-                s_table[d.slot] = part;
+                s_table[done.t] = part;
                 __threadfence_block();
-                complete = atomicAdd(&s_rowcnt[d.local_row], 1u) + 1u == (unsigned)share;
+                complete = atomicAdd(&s_rowcnt[done.local_row], 1u) + 1u == (unsigned)share;
             }
             complete = __shfl_sync(full, complete, 0);
             if (!complete) continue;
             __threadfence_block();
             RowEvent e;
-            e.row = d.row;
+            e.row = done.row;
             e.whole = share == nch;
             e.score = 0.f;
             e.argmax = 0;
-            e.first_slot = (int)(first_unit - lo);
-            e.first_chunk = (int)(first_unit - f * nch);
+            e.first_slot = (int)(first_unit - ulo);
+            e.first_chunk = (int)(first_unit - row_first);
             e.count = share;
             e.pad = 0;
             if (e.whole) fold_partials<KL>(s_table + e.first_slot, nch, e.score, e.argmax);
@@ -353,11 +337,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         }
     }
 
-    if (warp < kSStreamWarps && (!wait_ok || !queue_ok)) {
-        if (lane == 0 && p.status)
-            atomicCAS(p.status, 0u, (wait_ok ? kErrWaitQueue : kErrWaitPiece) | (blockIdx.x & 0xFF));
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // copies still in flight may land in the ring
-    }
+    if (warp < kSStreamWarps && !queue_ok && lane == 0 && p.status)
+        atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
 }
 
 }  // namespace ddv
