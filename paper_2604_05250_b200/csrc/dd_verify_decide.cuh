@@ -80,9 +80,16 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b, D
         int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
         if (staged) {
             const uint32_t bound = strictly ? cand : cand - 1u;      // cand >= 1 when not strict
+            if (nk <= 8) {
 #pragma unroll
-            for (int r = 0; r < kDecideKeys / 32; r += 4) {
-                c0 += kr[r] > bound; c1 += kr[r + 1] > bound; c2 += kr[r + 2] > bound; c3 += kr[r + 3] > bound;
+                for (int r = 0; r < 8; r += 4) {
+                    c0 += kr[r] > bound; c1 += kr[r + 1] > bound; c2 += kr[r + 2] > bound; c3 += kr[r + 3] > bound;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < kDecideKeys / 32; r += 4) {
+                    c0 += kr[r] > bound; c1 += kr[r + 1] > bound; c2 += kr[r + 2] > bound; c3 += kr[r + 3] > bound;
+                }
             }
         } else {
 #pragma unroll 4

@@ -87,12 +87,11 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     tally.b = -1;
     tally.target = 0;
     __shared__ float s_rehearsal[2];
-    if (warp == kSStreamWarps) {
-        // sequences without a single flagged row pass through; this CTA's share of them
+    // sequences without a single flagged row pass through; this CTA's share of them
+    auto pass_through = [&]() {
         for (int b = blockIdx.x; b < p.B; b += gridDim.x)
             if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
-    }
-
+    };
     bool rehearsed = false;
     bool queue_ok = true;
 
@@ -138,6 +137,15 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 fold_partials<KL>(fake, 32, sc, am);
                 if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
                 decide_sequence_rehearsal(p, &s_decide);
+                pass_through();
+            }
+            {
+                // the sequence this range ends in: its size is needed when its rows are counted
+                const int b_last = s_rows[(int)(f_hi - f_lo)] / p.P;
+                if (tally.b != b_last) {
+                    tally.b = b_last;
+                    tally.target = count_flagged(p, b_last);
+                }
             }
             unsigned int head = 0;
             for (unsigned idle = 0;;) {
@@ -337,6 +345,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         }
     }
 
+    if (warp == kSStreamWarps && !rehearsed) pass_through();      // this CTA had no range
     if (warp < kSStreamWarps && !queue_ok && lane == 0 && p.status)
         atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
 }

@@ -132,6 +132,17 @@ def test_degenerate_cases(dd, oracle_mod):
     compare(dd, oracle_mod, d1, v1, t1, f1, CONF, 0.5, 0, 0)
 
 
+def test_many_short_rows_and_long_sequences(dd, oracle_mod):
+    # more (row, chunk) units than the CTAs' tables hold at once (several rounds per CTA), and
+    # sequences longer than the decision stage keeps in shared memory
+    dra, ver, tokens, flags = synth.verify_inputs(15, 8192, 64, 5700, 0.2, seed=31)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 40, 3)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, CONF | PROB, 0.5, 7, 3)
+    # a sequence length between the two decision paths' limits
+    dra, ver, tokens, flags = synth.verify_inputs(2, 1500, 4104, 900, 0.2, seed=32)
+    compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 33, 1)
+
+
 def test_exact_ties_in_verifier_row(dd, oracle_mod):
     dra, ver, tokens, flags = synth.verify_inputs(1, 8, 20000, 8, 0.0, seed=13)
     top = synth.f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
