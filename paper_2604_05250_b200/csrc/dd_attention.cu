@@ -66,8 +66,8 @@ __device__ __forceinline__ void report(unsigned int *status, unsigned code)
     atomicCAS(status, 0u, code | (unsigned)(blockIdx.x & 0xFF));
 }
 
-// One key tile of the online softmax for one query row.  s[] holds the raw scores.
-// Returns the sum of the weights written; weights go to tensor memory as packed bf16.
+// One key tile of the online softmax for one query row; s[] holds the raw scores.
+// Row maximum of the raw scores (keys past the sequence end excluded).
 template <bool kMasked>
 __device__ __forceinline__ float row_max(const float (&s)[kBlockN], int valid)
 {
@@ -82,34 +82,46 @@ __device__ __forceinline__ float row_max(const float (&s)[kBlockN], int valid)
     return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
+// Weights P = 2^(s*c - m_ref) of the tile as packed bf16 into tensor memory, 32 keys (16
+// columns) at a time; returns the sum of the weights as rounded, and through mx the row
+// maximum of the raw scores seen on the way (so the caller can tell afterwards whether
+// m_ref was still a good reference point).  Two values per instruction where the
+// hardware has a packed form.
 template <bool kMasked>
-__device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int valid, float c, float neg_m,
-                                                 uint32_t tmem_p)
+__device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int valid, float c, float m_ref,
+                                                 uint32_t tmem_p, float &mx)
 {
-    float sum0 = 0.f, sum1 = 0.f;
+    const float2 c2 = make_float2(c, c), nm2 = make_float2(-m_ref, -m_ref);
+    float2 sum2 = make_float2(0.f, 0.f);
+    float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        uint32_t pk[32];
+    for (int q = 0; q < kBlockN / 32; ++q) {
+        uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 64; i += 2) {
-            const int e = h * 64 + i;
-            float p0 = ex2(fmaf(s[e], c, neg_m));
-            float p1 = ex2(fmaf(s[e + 1], c, neg_m));
+        for (int i = 0; i < 32; i += 2) {
+            const int e = q * 32 + i;
+            const float2 a = __ffma2_rn(make_float2(s[e], s[e + 1]), c2, nm2);
+            float p0 = ex2(a.x), p1 = ex2(a.y);
             if (kMasked) {
                 // keys past the end of the sequence get weight zero (a select, not -inf arithmetic: scale may be 0)
                 p0 = e < valid ? p0 : 0.f;
                 p1 = e + 1 < valid ? p1 : 0.f;
+                if (e < valid) m0 = fmaxf(m0, s[e]);
+                if (e + 1 < valid) m1 = fmaxf(m1, s[e + 1]);
+            } else {
+                m0 = fmaxf(m0, s[e]);
+                m1 = fmaxf(m1, s[e + 1]);
             }
             __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
             const uint32_t w = *reinterpret_cast<uint32_t *>(&b);
             pk[i / 2] = w;
             // the row sum takes the weights as rounded, so that O / l is an exact convex combination
-            sum0 += __uint_as_float(w << 16);
-            sum1 += __uint_as_float(w & 0xFFFF0000u);
+            sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)));
         }
-        tmem_st32(tmem_p + h * 32, pk);
+        tmem_st16(tmem_p + q * 16, pk);
     }
-    return sum0 + sum1;
+    mx = fmaxf(m0, m1);
+    return sum2.x + sum2.y;
 }
 
 template <int D>
@@ -188,30 +200,36 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
                 const int valid = p.N - j * kBlockN;       // keys of this tile that exist
                 const bool masked = valid < kBlockN;
-                const float mx = masked ? row_max<true>(s, valid) : row_max<false>(s, valid);
-                const float m_new = fmaxf(m_ref, mx * c);
-                const bool move = m_new > m_ref + kRescaleStep;   // always true on the first tile
+                // The first tile takes its reference point from its own maximum.  Later tiles are
+                // weighted against the reference point they inherit, in one pass, and only a row
+                // whose maximum turns out to have grown past it by more than the allowed step moves
+                // the reference point, rescales O and weights the tile again.
+                if (j == 0) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
+                float mx;
+                float sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
+                                   : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
+                const bool move = mx * c > m_ref + kRescaleStep;
                 if (__any_sync(0xffffffffu, move)) {
-                    const float alpha = move ? ex2(m_ref - m_new) : 1.f;
-                    if (move) m_ref = m_new;
+                    const float m_new = move ? mx * c : m_ref;
+                    const float alpha = ex2(m_ref - m_new);       // 1 where the row does not move
+                    m_ref = m_new;
                     l_run *= alpha;
-                    if (j > 0) {
-                        // O_g holds the sum over tiles < j once the previous P V has completed
-                        if (!mbar_wait(bar_o_full(g), (j - 1) & 1)) { err = kErrWaitO; break; }
-                        tc_fence_after();
+                    // O_g holds the sum over tiles < j once the previous P V has completed
+                    if (!mbar_wait(bar_o_full(g), (j - 1) & 1)) { err = kErrWaitO; break; }
+                    tc_fence_after();
 #pragma unroll
-                        for (int cb = 0; cb < D / 32; ++cb) {
-                            uint32_t r[32];
-                            tmem_ld32(tO + cb * 32, r);
-                            tmem_wait_ld();
+                    for (int cb = 0; cb < D / 32; ++cb) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + cb * 32, r);
+                        tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                            tmem_st32(tO + cb * 32, r);
-                        }
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(tO + cb * 32, r);
                     }
+                    tmem_wait_st();                               // the first weights are overwritten next
+                    sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
+                                 : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
                 }
-                const float sum = masked ? weights_to_tmem<true>(s, valid, c, -m_ref, tS)
-                                         : weights_to_tmem<false>(s, valid, c, -m_ref, tS);
                 l_run += sum;
                 tmem_wait_st();
                 tc_fence_before();
@@ -271,26 +289,31 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             // =============================================================== MMA issuer
             constexpr uint32_t kIdescS = idesc_bf16(kBlockM, kBlockN, false);
             constexpr uint32_t kIdescO = idesc_bf16(kBlockM, D, true);
+            // descriptors of a tile are the tile's base descriptor plus the byte offset / 16
+            const uint64_t desc_q0 = smem_desc_sw128(sQ, 16, 1024);
+            const uint64_t desc_k0 = smem_desc_sw128(sRing, 16, 1024);            // K-major operand (K tile)
+            const uint64_t desc_v0 = smem_desc_sw128(sRing, kBoxBytes, 1024);     // MN-major operand (V tile)
             unsigned err = 0;
             // S_g = Q_g K^T for the K tile in `slot`
             auto issue_s = [&](int g, int slot) {
-                const uint32_t a = sQ + g * kTileBytes, b = sRing + slot * kTileBytes;
+                const uint64_t a = desc_q0 + (uint64_t)(g * (kTileBytes >> 4));
+                const uint64_t b = desc_k0 + (uint64_t)(slot * (kTileBytes >> 4));
+                const uint32_t tS = tmem + kColS + g * kBlockN;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;   // 16 bf16 = 32 bytes per k-step
-                    mma_ss(tmem + kColS + g * kBlockN, smem_desc_sw128(a + off, 16, 1024),
-                           smem_desc_sw128(b + off, 16, 1024), kIdescS, ks > 0);
+                    const uint32_t off = ((ks / 4) * kBoxBytes + (ks % 4) * 32) >> 4;   // 16 bf16 = 32 bytes per k-step
+                    mma_ss(tS, a + off, b + off, kIdescS, ks > 0);
                 }
                 mma_commit(bar_s_full(g));
             };
             // O_g (+)= P_g V for the V tile in `slot`
             auto issue_o = [&](int g, int slot, bool first) {
-                const uint32_t b = sRing + slot * kTileBytes;
+                const uint64_t b = desc_v0 + (uint64_t)(slot * (kTileBytes >> 4));
+                const uint32_t tS = tmem + kColS + g * kBlockN, tO = tmem + kColO + g * D;
 #pragma unroll
                 for (int ks = 0; ks < kBlockN / 16; ++ks) {
                     // 16 keys = two 8-row groups of 1024 bytes; column blocks of 64 are one box apart
-                    mma_ts(tmem + kColO + g * D, tmem + kColS + g * kBlockN + ks * 8,
-                           smem_desc_sw128(b + ks * 2048, kBoxBytes, 1024), kIdescO, (!first || ks > 0));
+                    mma_ts(tO, tS + ks * 8, b + (uint32_t)(ks * (2048 >> 4)), kIdescO, (!first || ks > 0));
                 }
                 mma_commit(bar_o_full(g));
             };
