@@ -43,7 +43,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (None until a capture of that kernel exists).
-NCU_TRAFFIC_BYTES = {"attention": None, "verify": None}
+NCU_TRAFFIC_BYTES = {"attention": 25.27e6, "verify": 136.79e6}
 
 
 def attention_flops():
@@ -379,7 +379,7 @@ def run_ours(args):
                        "peak_used": f"{peaks['hbm']} GB/s ({peaks['source']})"},
         }
         if ver_step >= att_step:
-            roof = {"kernel": "verify_kernel", "bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm"], "unit": "GB/s",
+            roof = {"kernel": "verify_stream_kernel", "bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm"], "unit": "GB/s",
                     "frac": ver_gbs / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES["verify"], "peak_source": peaks["source"]}
         else:
             roof = {"kernel": "attention_kernel", "bound": "tensor", "achieved": att_tflops, "peak": att_peak,
