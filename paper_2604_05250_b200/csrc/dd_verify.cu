@@ -200,11 +200,31 @@ bool streaming_path(const void *drafter, const void *verifier, int V, bool kl)
     return (V % 8 == 0) && (((uintptr_t)verifier & 15) == 0) && (!kl || ((uintptr_t)drafter & 15) == 0);
 }
 
-void chunking(int V, bool streaming, int *nchunks, int *chunk)
+// Streaming path: pieces per chunk.  Every streaming warp of a CTA takes whole (row, chunk)
+// units in turn, so a CTA's time is rounds * pieces-per-unit; pick the unit size that wastes
+// least for `rows` flagged rows on `ctas` CTAs (a smaller unit only if it saves 5 %), among
+// those whose partials fit `max_partials` (0: no limit).
+int pick_pieces(int V, long rows, int ctas, long max_partials)
+{
+    int best = kMaxPiecesPerChunk;
+    long best_cost = -1;
+    for (int k = kMaxPiecesPerChunk; k >= kMinPiecesPerChunk; --k) {
+        const long nch = (V + (long)k * kPiece - 1) / ((long)k * kPiece);
+        if (max_partials > 0 && rows * nch > max_partials && k != kMaxPiecesPerChunk) continue;
+        const long per_cta = (rows * nch + ctas - 1) / ctas;
+        const long rounds = (per_cta + kSStreamWarps - 1) / kSStreamWarps;
+        const long cost = rounds * k;
+        // a finer cut has more chunk ends: it must save at least 5 % of the pieces
+        if (best_cost < 0 || cost * 20 <= best_cost * 19) { best_cost = cost; best = k; }
+    }
+    return best;
+}
+
+void chunking(int V, bool streaming, int pieces, int *nchunks, int *chunk)
 {
     if (streaming) {
-        *chunk = kSChunk;
-        *nchunks = (V + kSChunk - 1) / kSChunk;
+        *chunk = pieces * kPiece;
+        *nchunks = (V + *chunk - 1) / *chunk;
         return;
     }
     const int n = (V + kMaxChunk - 1) / kMaxChunk;
@@ -214,20 +234,24 @@ void chunking(int V, bool streaming, int *nchunks, int *chunk)
     *chunk = c;
 }
 
-template <bool KL>
-int launch_stream(const VerifyParams &p, cudaStream_t stream)
+// Number of SMs of the current device (cached), or a negative status.
+int sm_count_of_current_device()
 {
-    static bool attr_done[64] = {};
-    static int sm_count[64] = {};
+    static int cached[64] = {};
     int dev = 0;
     DD_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return dd::cuda_fail(cudaErrorInvalidDevice, "dd_verify: device index");
-    if (!attr_done[dev]) {
-        DD_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-        attr_done[dev] = true;
-    }
+    if (!cached[dev]) DD_CUDA_TRY(cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev));
+    return cached[dev];
+}
+
+template <bool KL>
+int launch_stream(const VerifyParams &p, cudaStream_t stream)
+{
+    const int sms = sm_count_of_current_device();
+    if (sms < 0) return sms;
     const long units = (long)p.B * p.P * p.nchunks;
-    const long grid = units < sm_count[dev] ? units : sm_count[dev];
+    const long grid = units < sms ? units : sms;
     verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, 0, stream>>>(p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
@@ -294,7 +318,7 @@ extern "C" size_t dd_verify_workspace_bytes(int B, int P, int V)
 {
     if (B <= 0 || P <= 0 || V <= 0) return 0;
     int nchunks, chunk;
-    chunking(V, V % 8 == 0, &nchunks, &chunk);
+    chunking(V, V % 8 == 0, kMinPiecesPerChunk, &nchunks, &chunk);       // the finest cut a launch may choose
     return workspace_bytes(B, P, nchunks) + counter_bytes(B, P);
 }
 
@@ -311,7 +335,13 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     const bool streaming = streaming_path(drafter_logits, verifier_logits, V, kl);
 
     VerifyParams p;
-    chunking(V, streaming, &p.nchunks, &p.chunk);
+    int pieces = kMaxPiecesPerChunk;
+    if (streaming) {
+        const int sms = sm_count_of_current_device();
+        if (sms < 0) return sms;
+        pieces = pick_pieces(V, (long)B * P, sms, (1L << 31) - 1);
+    }
+    chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
     if ((long)B * P * p.nchunks >= (1L << 31)) return DD_ERR_UNSUPPORTED;
 
     dd::DeviceCtx *ctx = dd::current_ctx();
@@ -395,10 +425,18 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     const bool streaming = streaming_path(drafter_logits, verifier_logits, V, kl);
 
     VerifyParams p;
-    chunking(V, streaming, &p.nchunks, &p.chunk);
-    // the fixed scratch bounds the problem size (checked against the finer of the two chunkings)
-    const long worst_chunks = (V + kSChunk - 1) / kSChunk;
-    if ((long)B * P > kStaticMaxRows || (long)B * P * worst_chunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
+    // the fixed scratch bounds the problem size (stated for chunks of 8192 logits; a finer cut is
+    // only chosen where its partials still fit)
+    const long coarse_chunks = (V + kSChunk - 1) / kSChunk;
+    if ((long)B * P > kStaticMaxRows || (long)B * P * coarse_chunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
+    int pieces = kMaxPiecesPerChunk;
+    if (streaming) {
+        const int sms = sm_count_of_current_device();
+        if (sms < 0) return sms;
+        pieces = pick_pieces(V, (long)B * P, sms, kStaticMaxPartials);
+    }
+    chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
+    if ((long)B * P * p.nchunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
 
     int dev = -1;
     DD_CUDA_TRY(cudaGetDevice(&dev));

@@ -1,7 +1,8 @@
 // Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
 //
 // One persistent CTA per SM: fifteen warps stream, one warp publishes.  The flagged rows'
-// (row, chunk) units, 8192 logits each, are numbered in row order and cut into equal
+// (row, chunk) units (3 to 8 pieces of 1024 logits, chosen per launch so that the units of a
+// range come out in whole rounds of the streaming warps) are numbered in row order and cut into equal
 // contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  The
 // range's units go to the streaming warps in turn.  A warp walks its unit in pieces of 1024
 // logits per tensor: every lane holds four 16-byte vectors per tensor of the current piece
@@ -28,8 +29,8 @@ constexpr int kSWarps = kSStreamWarps + 1;                    // + one that publ
 constexpr int kSThreads = kSWarps * 32;
 constexpr int kSQueue = 64;                                   // finished-chunk queue slots
 constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per step of a warp
-constexpr int kPiecesPerChunk = 8;
-constexpr int kSChunk = kPiece * kPiecesPerChunk;             // 8192 logits per (row, chunk)
+constexpr int kMinPiecesPerChunk = 3, kMaxPiecesPerChunk = 8; // a (row, chunk) unit is 3072 .. 8192 logits
+constexpr int kSChunk = kPiece * kMaxPiecesPerChunk;
 constexpr int kSTable = 768;                                  // chunk partials a CTA keeps per range
 constexpr unsigned kErrWaitQueue = 0x800;
 

@@ -224,7 +224,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
 
         // =================================================================== streaming warps
         const unsigned ulo = (unsigned)lo, uhi = (unsigned)hi, uflo = (unsigned)f_lo;   // units fit 31 bits
-        const int last_pieces = (p.V - (nch - 1) * kSChunk + kPiece - 1) / kPiece;       // of a row's last chunk
+        const int chunk_len = p.chunk, chunk_pieces = p.chunk / kPiece;                 // logits, pieces per chunk
+        const int last_pieces = (p.V - (nch - 1) * chunk_len + kPiece - 1) / kPiece;       // of a row's last chunk
 
         // Units of the range go to the streaming warps in turn: warp w takes units w, w + 15, ...
         // A cursor walks one warp's pieces in order (all lanes hold the same values).
@@ -235,7 +236,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         };
         auto enter_unit = [&](Cursor &c) {
             if (c.t >= n_units) return;
-            c.npieces = c.chunk == nch - 1 ? last_pieces : kPiecesPerChunk;
+            c.npieces = c.chunk == nch - 1 ? last_pieces : chunk_pieces;
             c.row = s_rows[c.local_row];
         };
         auto advance = [&](Cursor &c) {
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         };
         // the lane's vectors of the cursor's piece: four per tensor, -inf where the row has ended
         auto fetch = [&](const Cursor &c, uint4 (&v)[kVecPerThread], uint4 (&d)[kVecPerThread]) {
-            const int e_begin = c.chunk * kSChunk + c.piece * kPiece;
+            const int e_begin = c.chunk * chunk_len + c.piece * kPiece;
             const int n = p.V - e_begin;                      // logits left in the row
             const size_t off = (size_t)c.row * p.V + e_begin;
             const uint4 *gv = reinterpret_cast<const uint4 *>(p.verifier + off) + lane;
@@ -303,7 +304,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             advance(nc);
             if (nc.t < n_units) fetch(nc, nv, nd);            // in flight while this piece is computed
 
-            const int n = min(kPiece, p.V - (cc.chunk * kSChunk + cc.piece * kPiece));
+            const int n = min(kPiece, p.V - (cc.chunk * chunk_len + cc.piece * kPiece));
             if (n == kPiece) lane_piece<KL, true>(L, rv, rd, n, lane, cc.piece);
             else lane_piece<KL, false>(L, rv, rd, n, lane, cc.piece);
             const bool chunk_ends = cc.piece == cc.npieces - 1;
@@ -313,7 +314,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
 
             // ---- the chunk is complete: into the table; the warp that completes the range's share
             // of a row hands the row on
-            const Partial part = lanes_to_partial<KL>(L, done.chunk * kSChunk, lane);
+            const Partial part = lanes_to_partial<KL>(L, done.chunk * chunk_len, lane);
             lane_reset(L);
             const unsigned row_first = (uflo + (unsigned)done.local_row) * (unsigned)nch;   // the row's unit 0
             const unsigned first_unit = max(ulo, row_first), end_unit = min(uhi, row_first + (unsigned)nch);
