@@ -55,8 +55,8 @@ struct Smem {
     static constexpr int kQ = 0;                                   // two query tiles
     static constexpr int kRing = kQTiles * kTileBytes;             // kStages K/V tiles
     static constexpr int kBars = kRing + kStages * kTileBytes;
-    // barriers (8 bytes each): q_full, kv_full[kStages], kv_empty[kStages], s_full[2], p_full[2], o_full[2]
-    static constexpr int kNumBars = 1 + 2 * kStages + 6;
+    // barriers (8 bytes each): q_full[2], kv_full[kStages], kv_empty[kStages], s_full[2], p_full[2], o_full[2]
+    static constexpr int kNumBars = 2 + 2 * kStages + 6;
     static constexpr int kTmemSlot = kBars + 8 * kNumBars;
     static constexpr int kTotal = kTmemSlot + 16;
 };
@@ -136,12 +136,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     constexpr uint32_t kTileBytes = Smem<D>::kTileBytes;
     const uint32_t sQ = smem_base + Smem<D>::kQ, sRing = smem_base + Smem<D>::kRing;
     const uint32_t bars = smem_base + Smem<D>::kBars;
-    const uint32_t bar_q = bars;
-    auto bar_kv_full = [&](int s) { return bars + 8u * (1 + s); };
-    auto bar_kv_empty = [&](int s) { return bars + 8u * (1 + kStages + s); };
-    auto bar_s_full = [&](int g) { return bars + 8u * (1 + 2 * kStages + g); };
-    auto bar_p_full = [&](int g) { return bars + 8u * (3 + 2 * kStages + g); };
-    auto bar_o_full = [&](int g) { return bars + 8u * (5 + 2 * kStages + g); };
+    auto bar_q = [&](int g) { return bars + 8u * g; };
+    auto bar_kv_full = [&](int s) { return bars + 8u * (2 + s); };
+    auto bar_kv_empty = [&](int s) { return bars + 8u * (2 + kStages + s); };
+    auto bar_s_full = [&](int g) { return bars + 8u * (2 + 2 * kStages + g); };
+    auto bar_p_full = [&](int g) { return bars + 8u * (4 + 2 * kStages + g); };
+    auto bar_o_full = [&](int g) { return bars + 8u * (6 + 2 * kStages + g); };
     const uint32_t tmem_slot = smem_base + Smem<D>::kTmemSlot;
     volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + Smem<D>::kTmemSlot);
 
@@ -157,7 +157,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     if (tid == 0) {
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-        mbar_init(bar_q, 1);
+        mbar_init(bar_q(0), 1); mbar_init(bar_q(1), 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
         for (int g = 0; g < kQTiles; ++g) {
             mbar_init(bar_s_full(g), 1);
@@ -269,13 +269,17 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         reg_dec<72>();
         if (warp == kLoadWarp && lane == 0) {
             // =============================================================== TMA producer
-            mbar_expect_tx(bar_q, ntiles * kTileBytes);
-            for (int g = 0; g < ntiles; ++g)
+            // what the first MMA needs comes first: Q tile 0, K tile 0, then Q tile 1
+            auto load_q = [&](int g) {
+                mbar_expect_tx(bar_q(g), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_load_3d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q, cx * 64, row0 + g * kBlockM, bh);
+                    tma_load_3d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM, bh);
+            };
+            load_q(0);
             // ring items: 2j = K tile j, 2j+1 = V tile j
             for (int item = 0; item < 2 * nkv; ++item) {
+                if (item == 1 && ntiles > 1) load_q(1);
                 const int slot = item % kStages, use = item / kStages;
                 if (use > 0 && !mbar_wait(bar_kv_empty(slot), (use - 1) & 1)) { report(p.status, kErrWaitSlot); break; }
                 const uint32_t dst = sRing + slot * kTileBytes;
@@ -321,10 +325,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 return mbar_wait(bar_kv_full(item % kStages), (item / kStages) & 1);
             };
             do {
-                if (!mbar_wait(bar_q, 0)) { err = kErrWaitQ; break; }
+                if (!mbar_wait(bar_q(0), 0)) { err = kErrWaitQ; break; }
                 if (!wait_item(0)) { err = kErrWaitKV; break; }
                 tc_fence_after();
-                for (int g = 0; g < ntiles; ++g) issue_s(g, 0);
+                issue_s(0, 0);
+                if (ntiles > 1) {
+                    if (!mbar_wait(bar_q(1), 0)) { err = kErrWaitQ; break; }
+                    tc_fence_after();
+                    issue_s(1, 0);
+                }
                 mma_commit(bar_kv_empty(0));
                 for (int j = 0; j < nkv && err == 0; ++j) {
                     const int item_v = 2 * j + 1, item_k = 2 * j + 2;
