@@ -141,6 +141,16 @@ def graph_chunk(K, cap=200):
     return g
 
 
+def max_over_ranks(values, device, distributed):
+    """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest rank)."""
+    import torch
+    vals = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if distributed:
+        import torch.distributed as dist
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    return [float(x) for x in vals.tolist()]
+
+
 def bf16_tensor(bits, device=None, pin=False):
     import torch
     t = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
@@ -358,10 +368,7 @@ def run_ours(args):
     assert dd.attention_status() == 0
 
     # ---- max over ranks
-    vals = torch.tensor([total_ms, att_ms, ver_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if distributed:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    total_ms, att_ms, ver_ms, e2e_ms = (float(x) for x in vals.tolist())
+    total_ms, att_ms, ver_ms, e2e_ms = max_over_ranks([total_ms, att_ms, ver_ms, e2e_ms], dev, distributed)
     ms_step, att_step, ver_step = total_ms / K, att_ms / K, ver_ms / K
 
     if rank == 0:
