@@ -178,7 +178,7 @@ def cpu_baseline(oracle, att_in, ver_in, budget_s=12.0):
     att_rows = np.arange(ATT["N"], dtype=np.int32)
     times = []
     t_start = time.perf_counter()
-    while not times or (time.perf_counter() - t_start < budget_s and len(times) < 8):
+    while not times or (time.perf_counter() - t_start < budget_s and len(times) < 64):
         times.append(oracle_step_sample(oracle, att_in, ver_in, att_rows, VER["P"]))
     return {"value": 1e3 * float(np.mean(times)), "unit": "ms", "cores": oracle.threads(), "kind": "oracle",
             "sample": f"the full cfg1 step (all {ATT['H']}x{ATT['N']} attention rows, all {VER['P']} logit rows), "

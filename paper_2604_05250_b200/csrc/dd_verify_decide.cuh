@@ -26,8 +26,22 @@ struct __align__(16) DecideStage {      // one per deciding warp, in shared memo
     int32_t top[kDecideKeys];      // verifier argmax of position i
 };
 
-__device__ __noinline__ void decide_sequence_impl(const VerifyParams p, int b, DecideStage *stage, bool dry)
+__device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int b, DecideStage *stage, bool dry)
 {
+    // Every field goes into a register once: the stores below are through generic pointers, after
+    // which the compiler would have to read the by-value structure again.
+    struct {
+        const uint8_t *flags; const int32_t *tokens; const float *row_score; const int *row_argmax;
+        int32_t *out_tokens; uint8_t *out_mask; float *out_score;
+        int P, k, algo, probabilistic, emit_drafter;
+        float tau;
+        uint32_t seed_lo, seed_hi;
+    } p;
+    p.flags = params.flags; p.tokens = params.tokens; p.row_score = params.row_score; p.row_argmax = params.row_argmax;
+    p.out_tokens = params.out_tokens; p.out_mask = params.out_mask; p.out_score = params.out_score;
+    p.P = params.P; p.k = params.k; p.algo = params.algo; p.probabilistic = params.probabilistic;
+    p.emit_drafter = params.emit_drafter; p.tau = params.tau; p.seed_lo = params.seed_lo; p.seed_hi = params.seed_hi;
+
     const int lane = threadIdx.x & 31;
     const unsigned full = 0xFFFFFFFFu;
     const long base = (long)b * p.P;
