@@ -127,7 +127,8 @@ __device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                 const AttnParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
     // 128-byte-swizzled tiles must start on a 1024-byte boundary
@@ -156,7 +157,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     constexpr uint32_t kColS = 0, kColO = 256;
 
     if (tid == 0) {
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_o);
         mbar_init(bar_q(0), 1); mbar_init(bar_q(1), 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
         for (int g = 0; g < kQTiles; ++g) {
@@ -237,32 +238,44 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             if (err == 0 && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
             if (err == 0) {
-                // ---- epilogue: O / l -> bf16 -> global
+                // ---- epilogue: O / l -> bf16 -> this tile's Q buffer (every MMA that read it has
+                // completed), in the swizzled layout of the tensor map, -> global by TMA (rows past N
+                // are clipped by the map)
                 tc_fence_after();
-                const int row = row0 + g * kBlockM + (warp & 3) * 32 + lane;
+                const int r = (warp & 3) * 32 + lane;                 // row within the tile
                 const float inv = 1.f / l_run;
-                __nv_bfloat16 *dst = p.out + ((size_t)bh * p.N + row) * D;
+                const uint32_t stage = sQ + g * kTileBytes + r * 128;
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
-                    uint32_t r[32];
-                    tmem_ld32(tO + cb * 32, r);
+                    uint32_t acc[32];
+                    tmem_ld32(tO + cb * 32, acc);
                     tmem_wait_ld();
-                    if (row < p.N) {
+                    const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
 #pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
-                            uint32_t w[4];
+                    for (int i = 0; i < 32; i += 8) {
+                        uint32_t w[4];
 #pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * h]) * inv,
-                                                                         __uint_as_float(r[i + 2 * h + 1]) * inv);
-                                w[h] = *reinterpret_cast<uint32_t *>(&v);
-                            }
-                            *reinterpret_cast<uint4 *>(dst + cb * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+                        for (int h = 0; h < 4; ++h) {
+                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * inv,
+                                                                     __uint_as_float(acc[i + 2 * h + 1]) * inv);
+                            w[h] = *reinterpret_cast<uint32_t *>(&v);
                         }
+                        const int chunk = (cb % 2) * 4 + i / 8;         // 16-byte chunk of the 128-byte row
+                        st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
                     }
                 }
+                fence_proxy_async_smem();
             } else {
                 report(p.status, err);
+            }
+            // every thread of the warpgroup comes here, also after an expired wait
+            named_bar_sync(1 + g, kBlockM);
+            if (err == 0 && (warp & 3) == 0 && lane == 0) {
+#pragma unroll
+                for (int cx = 0; cx < kBoxes; ++cx)
+                    tma_store_3d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, bh);
+                tma_store_commit();
+                tma_store_wait_read();
             }
         }
     } else {
@@ -405,7 +418,8 @@ int make_tmap(CUtensorMap *m, const void *base, int BH, int N, int D)
 }
 
 template <int D>
-int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const AttnParams &p, cudaStream_t s)
+int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
+           const AttnParams &p, cudaStream_t s)
 {
     static bool attr_done[64] = {};
     int dev = 0;
@@ -416,7 +430,7 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
         attr_done[dev] = true;
     }
     const long grid = (long)p.BH * p.m_blocks;
-    attention_kernel<D><<<(unsigned)grid, kThreads, smem, s>>>(tq, tk, tv, p);
+    attention_kernel<D><<<(unsigned)grid, kThreads, smem, s>>>(tq, tk, tv, to, p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
     return DD_OK;
@@ -441,11 +455,12 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
         DD_CUDA_TRY(cudaMalloc(&ctx->attn_status, 256));
         DD_CUDA_TRY(cudaMemset(ctx->attn_status, 0, 256));
     }
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     int rc;
     if ((rc = make_tmap(&tq, q, (int)BH, N, D)) != DD_OK) return rc;
     if ((rc = make_tmap(&tk, k, (int)BH, N, D)) != DD_OK) return rc;
     if ((rc = make_tmap(&tv, v, (int)BH, N, D)) != DD_OK) return rc;
+    if ((rc = make_tmap(&to, out, (int)BH, N, D)) != DD_OK) return rc;
 
     AttnParams p;
     p.out = (__nv_bfloat16 *)out;
@@ -454,7 +469,7 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->attn_status;
     cudaStream_t s = (cudaStream_t)stream;
-    return D == 64 ? launch<64>(tq, tk, tv, p, s) : launch<128>(tq, tk, tv, p, s);
+    return D == 64 ? launch<64>(tq, tk, tv, to, p, s) : launch<128>(tq, tk, tv, to, p, s);
 }
 
 }  // namespace
