@@ -211,9 +211,23 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
     }
 }
 
+}  // namespace ddv
+
+#include "dd_verify_decide_small.cuh"
+
+namespace ddv {
+
+// Short sequences are decided from registers, longer ones from the staging area.
+__device__ __forceinline__ void decide_dispatch(const VerifyParams &p, int b, DecideStage *stage, bool dry)
+{
+    if (p.P <= 256) decide_sequence_small<8>(p, b, dry);
+    else if (p.P <= 512) decide_sequence_small<16>(p, b, dry);
+    else decide_sequence_impl(p, b, stage, dry);
+}
+
 __device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b, DecideStage *stage)
 {
-    decide_sequence_impl(p, b, stage, false);
+    decide_dispatch(p, b, stage, false);
 }
 
 // Runs the decision code on sequence 0 without storing anything.  The decision runs once per
@@ -221,7 +235,7 @@ __device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b, De
 // cache; a warp with nothing to do yet calls this to bring them back in.
 __device__ __forceinline__ void decide_sequence_rehearsal(const VerifyParams &p, DecideStage *stage)
 {
-    decide_sequence_impl(p, 0, stage, true);
+    decide_dispatch(p, 0, stage, true);
 }
 
 // One sequence has one more completed row; the warp that completes the sequence decides it.
