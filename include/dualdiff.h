@@ -108,8 +108,34 @@ int dd_verify(const void *drafter_logits, const void *verifier_logits,
               int32_t *out_tokens, uint8_t *out_mask, float *out_score,
               int B, int P, int V, void *stream);
 
+/* `layout` argument of dd_block_attention. */
+enum {
+    DD_LAYOUT_BHND = 0, /* q, out [B,H,Nq,D]; k, v [B,H,Nkv,D]                     */
+    DD_LAYOUT_BNHD = 1  /* q, out [B,Nq,H,D]; k, v [B,Nkv,H,D] (heads interleaved) */
+};
+
 /*
- * Host-buffer forms of the two calls above (same definitions, same errors).
+ * Attention of a block of queries over cached keys and values (Section 2.2,
+ * Eq. 3 as written: the queries of the positions being computed against the
+ * stored K and V of the whole context; the shape of the drafter's step with a
+ * block-wise KV cache, Section 2.3).  No mask among the valid keys:
+ *     out[b,h,i,:] = sum_{j < n_b} softmax_j(scale * q[b,h,i,:] . k[b,h,j,:]) v[b,h,j,:]
+ * for i in [0,Nq), where n_b = Nkv if kv_len is NULL, else kv_len[b] clamped to
+ * [0,Nkv] (keys at and beyond n_b are padding and never contribute).  A
+ * sequence with n_b = 0 gets out = 0.  dd_bidir_attention is the case
+ * Nq = Nkv, kv_len = NULL, DD_LAYOUT_BHND, and runs the same kernel.
+ * q, k, v, out: bf16 in the given layout, D innermost, contiguous, 16-byte
+ * aligned, out not overlapping the inputs; kv_len: int32 [B] DEVICE pointer or
+ * NULL, read by the kernel when it runs.
+ * Supported and errors: as dd_bidir_attention, with Nq, Nkv >= 1;
+ * DD_ERR_INVALID_ARG for an unknown layout.
+ */
+int dd_block_attention(const void *q, const void *k, const void *v, void *out,
+                       int B, int H, int Nq, int Nkv, int D,
+                       const int32_t *kv_len, int layout, float scale, void *stream);
+
+/*
+ * Host-buffer forms of dd_bidir_attention and dd_verify (same definitions, same errors).
  * Every pointer is a HOST pointer.  The call enqueues, on `stream`, the
  * host-to-device copies into library-owned staging memory, the kernel, and the
  * device-to-host copies of the outputs; the outputs are valid once the stream

@@ -44,6 +44,8 @@ def _load():
         lib.dd_oracle_attention.restype = None
         lib.dd_oracle_attention_probs.argtypes = [vp, vp, i32, i32, i32, f64, i32, i32, i32, vp]
         lib.dd_oracle_attention_probs.restype = None
+        lib.dd_oracle_block_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, f64, vp]
+        lib.dd_oracle_block_attention.restype = None
         lib.dd_oracle_philox4x32_10.argtypes = [vp, vp, vp]
         lib.dd_oracle_philox4x32_10.restype = None
         lib.dd_oracle_uniform.argtypes = [u64, i32, i32]
@@ -94,6 +96,33 @@ def attention(q, k, v, scale, rows=None, return_lse=False):
                                 _ptr(rows), 0 if rows is None else rows.size,
                                 _ptr(out), _ptr(lse))
     return (out, lse) if return_lse else out
+
+
+def block_attention(q, k, v, scale, kv_len=None, layout="bhnd"):
+    """Eq. 3 for a block of queries over stored keys (Section 2.3's cached drafter step).
+
+    layout "bhnd": q [B,H,Nq,D], k,v [B,H,Nkv,D]; "bnhd": q [B,Nq,H,D], k,v [B,Nkv,H,D]
+    (uint16 bf16 bits).  kv_len: int32 [B] valid keys per sequence, or None.
+    Returns float64 in the layout of q."""
+    assert layout in ("bhnd", "bnhd")
+    q = _u16(q)
+    k = _u16(k)
+    if layout == "bhnd":
+        B, H, Nq, D = q.shape
+        Nkv = k.shape[2]
+        assert k.shape == (B, H, Nkv, D)
+    else:
+        B, Nq, H, D = q.shape
+        Nkv = k.shape[1]
+        assert k.shape == (B, Nkv, H, D)
+    v = _u16(v, k.shape)
+    if kv_len is not None:
+        kv_len = np.ascontiguousarray(kv_len, dtype=np.int32)
+        assert kv_len.shape == (B,)
+    out = np.empty(q.shape, dtype=np.float64)
+    _load().dd_oracle_block_attention(_ptr(q), _ptr(k), _ptr(v), B, H, Nq, Nkv, D, _ptr(kv_len),
+                                      1 if layout == "bhnd" else 0, float(scale), _ptr(out))
+    return out
 
 
 def attention_probs(q, k, scale, b, h, i):

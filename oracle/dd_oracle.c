@@ -18,6 +18,9 @@
  *   dd_oracle_attention        pinned   (softmax rows sum to 1, constant V,
  *                                        key permutation, N=1, zero keys,
  *                                        one-hot limit, scipy fp64 softmax)
+ *   dd_oracle_block_attention  pinned   (numpy fp64 softmax on the valid keys,
+ *                                        truncation to kv_len, layout transpose,
+ *                                        one key, constant V, zero keys)
  *   dd_oracle_row_scores       pinned   (KL(p,p)=0, KL>=0, two-token closed
  *                                        form, constant logits, shift
  *                                        invariance, scipy rel_entr)
@@ -126,6 +129,65 @@ void dd_oracle_attention_probs(const uint16_t *q, const uint16_t *k,
         denom += p[j];
     }
     for (int j = 0; j < N; ++j) p[j] /= denom;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Attention of a block of queries over stored keys and values: Eq. 3 as it is
+ * written (queries of the positions being computed, keys and values of the
+ * context), the shape of a drafter step with a block-wise KV cache
+ * (Section 2.3):
+ *     z_i = softmax_{j < n_b}( scale * q_i . k_j ) V ,   i = 0..Nq-1,
+ * n_b = kv_len[b] clamped to [0,Nkv] (Nkv if kv_len is NULL); keys at and
+ * beyond n_b are padding.  n_b = 0 gives z = 0.
+ *
+ * head_major = 1: q [B,H,Nq,D], k,v [B,H,Nkv,D]; 0: q [B,Nq,H,D], k,v [B,Nkv,H,D].
+ * out: fp64 in the layout of q.                                              */
+static size_t elem_index(int head_major, int H, int N, int D, int b, int h, int n, int d)
+{
+    return head_major ? (((size_t)b * H + h) * N + n) * D + d
+                      : (((size_t)b * N + n) * H + h) * D + d;
+}
+
+void dd_oracle_block_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                               int B, int H, int Nq, int Nkv, int D,
+                               const int32_t *kv_len, int head_major, double scale,
+                               double *out)
+{
+    const long total = (long)B * H * Nq;
+#pragma omp parallel
+    {
+        double *w = (double *)malloc(sizeof(double) * (size_t)Nkv);
+#pragma omp for schedule(dynamic, 16)
+        for (long t = 0; t < total; ++t) {
+            const int b = (int)(t / ((long)H * Nq));
+            const int h = (int)((t / Nq) % H);
+            const int i = (int)(t % Nq);
+            int n = kv_len ? kv_len[b] : Nkv;
+            if (n < 0) n = 0;
+            if (n > Nkv) n = Nkv;
+            double m = -INFINITY;
+            for (int j = 0; j < n; ++j) {
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d)
+                    dot += bf16_to_f64(q[elem_index(head_major, H, Nq, D, b, h, i, d)]) *
+                           bf16_to_f64(k[elem_index(head_major, H, Nkv, D, b, h, j, d)]);
+                w[j] = scale * dot;
+                if (w[j] > m) m = w[j];
+            }
+            double denom = 0.0;
+            for (int j = 0; j < n; ++j) {
+                w[j] = exp(w[j] - m);
+                denom += w[j];
+            }
+            for (int d = 0; d < D; ++d) {
+                double acc = 0.0;
+                for (int j = 0; j < n; ++j)
+                    acc += w[j] * bf16_to_f64(v[elem_index(head_major, H, Nkv, D, b, h, j, d)]);
+                out[elem_index(head_major, H, Nq, D, b, h, i, d)] = n > 0 ? acc / denom : 0.0;
+            }
+        }
+        free(w);
+    }
 }
 
 /* ------------------------------------------------------------------------ */

@@ -17,10 +17,11 @@ LIB_PATH = os.path.join(_HERE, "libdualdiff.so")
 DD_OK, DD_ERR_INVALID_ARG, DD_ERR_UNSUPPORTED, DD_ERR_CUDA, DD_ERR_TIMEOUT = 0, -1, -2, -3, -4
 DD_MODE_TRUST, DD_MODE_KL, DD_MODE_CONF = 0, 1, 2
 DD_FLAG_PROBABILISTIC, DD_FLAG_EMIT_DRAFTER = 0x100, 0x200
+DD_LAYOUT_BHND, DD_LAYOUT_BNHD = 0, 1
 
 # every symbol include/dualdiff.h declares
 EXPORTS = (
-    "dd_bidir_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
+    "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
     "dd_status_string", "dd_last_cuda_error", "dd_version",
 )
@@ -49,6 +50,8 @@ def lib() -> ctypes.CDLL:
         ver = [vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, vp]
         L.dd_bidir_attention.argtypes = attn
         L.dd_bidir_attention_host.argtypes = attn
+        L.dd_block_attention.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, f32, vp]
+        L.dd_block_attention.restype = i32
         L.dd_verify.argtypes = ver
         L.dd_verify_host.argtypes = ver
         L.dd_verify_static.argtypes = ver
@@ -118,6 +121,39 @@ def bidir_attention(q, k, v, out=None, scale=None, stream=None, host=False):
         scale = float(D) ** -0.5
     fn = lib().dd_bidir_attention_host if host else lib().dd_bidir_attention
     _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale), _stream_ptr(stream)))
+    return out
+
+
+def block_attention(q, k, v, kv_len=None, layout="bhnd", out=None, scale=None, stream=None):
+    """dd_block_attention: a block of Nq queries over Nkv stored keys and values.
+
+    layout "bhnd": q [B,H,Nq,D], k, v [B,H,Nkv,D]; "bnhd": q [B,Nq,H,D], k, v [B,Nkv,H,D];
+    torch.bfloat16 device tensors.  kv_len: int32 [B] device tensor (valid keys per sequence)
+    or None.  Returns out (allocated if None), in the layout of q."""
+    import torch
+    if layout == "bhnd":
+        B, H, Nq, D = q.shape
+        Nkv = k.shape[2]
+        kshape = (B, H, Nkv, D)
+    elif layout == "bnhd":
+        B, Nq, H, D = q.shape
+        Nkv = k.shape[1]
+        kshape = (B, Nkv, H, D)
+    else:
+        raise ValueError("layout: 'bhnd' or 'bnhd'")
+    _require(q, torch.bfloat16, tuple(q.shape), True, "q")
+    _require(k, torch.bfloat16, kshape, True, "k")
+    _require(v, torch.bfloat16, kshape, True, "v")
+    if kv_len is not None:
+        _require(kv_len, torch.int32, (B,), True, "kv_len")
+    if out is None:
+        out = torch.empty_like(q)
+    _require(out, torch.bfloat16, tuple(q.shape), True, "out")
+    if scale is None:
+        scale = float(D) ** -0.5
+    _check(lib().dd_block_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, Nq, Nkv, D, _ptr(kv_len),
+                                    DD_LAYOUT_BHND if layout == "bhnd" else DD_LAYOUT_BNHD, float(scale),
+                                    _stream_ptr(stream)))
     return out
 
 

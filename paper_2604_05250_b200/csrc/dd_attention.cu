@@ -1,12 +1,15 @@
 // dd_bidir_attention: full-sequence bidirectional attention (Section 2.2; Eq. 3
-// evaluated over the whole key range) for sm_100a.
+// evaluated over the whole key range) for sm_100a, and dd_block_attention: the same
+// equation for a block of Nq queries against Nkv (cached) keys, with a per-sequence
+// number of valid keys and either memory layout.  One kernel serves both.
 //
 // One CTA owns two tiles of 128 query rows of one (batch, head) and walks over
 // the keys in tiles of 128.  The CTA is warp-specialised:
 //   warps 0-3   softmax of query tile 0 (thread = query row = TMEM lane)
 //   warps 4-7   softmax of query tile 1
-//   warp  8     one thread feeds a ring of K/V tiles by TMA (3-D tensor maps over
-//               [B*H, N, D], 128-byte swizzle; rows past N read as zero)
+//   warp  8     one thread feeds a ring of K/V tiles by TMA (4-D tensor maps over
+//               (D, N, H, B) with the strides of the layout, 128-byte swizzle; rows
+//               past N read as zero)
 //   warp  9     one thread issues every tcgen05 MMA
 // S_g = Q_g K^T goes to tensor memory; the softmax thread reads its row, keeps the
 // running maximum and sum in fp32 (online softmax in base 2, scale*log2e folded
@@ -42,9 +45,9 @@ enum : unsigned { kErrWaitQ = 0x100, kErrWaitKV = 0x200, kErrWaitS = 0x300, kErr
                   kErrWaitP = 0x500, kErrWaitSlot = 0x600 };
 
 struct AttnParams {
-    __nv_bfloat16 *out;
-    int BH, N, D;
-    int m_blocks;              // CTAs per (batch, head) = ceil(N / 256)
+    int BH, H, Nq, Nkv, D;
+    int m_blocks;              // CTAs per (batch, head) = ceil(Nq / 256)
+    const int *kv_len;         // [B] keys of each sequence that exist (clamped to 0..Nkv), or null: Nkv
     float scale_log2;          // scale * log2(e)
     unsigned int *status;
 };
@@ -150,8 +153,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int bh = blockIdx.x / p.m_blocks;
     const int mb = blockIdx.x - bh * p.m_blocks;
     const int row0 = mb * (kQTiles * kBlockM);
-    const int nkv = (p.N + kBlockN - 1) / kBlockN;
-    const int ntiles = (p.N - row0 > kBlockM) ? 2 : 1;    // query tiles of this CTA that hold rows
+    const int b_idx = bh / p.H, h_idx = bh - b_idx * p.H;
+    const int keys = p.kv_len ? min(max(p.kv_len[b_idx], 0), p.Nkv) : p.Nkv;   // keys that exist
+    const int nkv = (keys + kBlockN - 1) / kBlockN;       // 0: the sequence has no key, the output is zero
+    const int ntiles = (p.Nq - row0 > kBlockM) ? 2 : 1;   // query tiles of this CTA that hold rows
     constexpr int kBoxes = D / 64;                 // 64-column (128-byte) boxes per tile row
     constexpr uint32_t kBoxBytes = 128 * 128;      // 128 rows x 128 bytes
     constexpr uint32_t kColS = 0, kColO = 256;
@@ -199,7 +204,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     tmem_ld32(tS + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cb * 32]));
                 tmem_wait_ld();
 
-                const int valid = p.N - j * kBlockN;       // keys of this tile that exist
+                const int valid = keys - j * kBlockN;      // keys of this tile that exist
                 const bool masked = valid < kBlockN;
                 // The first tile takes its reference point from its own maximum.  Later tiles are
                 // weighted against the reference point they inherit, in one pass, and only a row
@@ -236,20 +241,25 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 tc_fence_before();
                 mbar_arrive(bar_p_full(g));
             }
-            if (err == 0 && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
+            if (err == 0 && nkv > 0 && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
             if (err == 0) {
                 // ---- epilogue: O / l -> bf16 -> this tile's Q buffer (every MMA that read it has
                 // completed), in the swizzled layout of the tensor map, -> global by TMA (rows past N
                 // are clipped by the map)
                 tc_fence_after();
                 const int r = (warp & 3) * 32 + lane;                 // row within the tile
-                const float inv = 1.f / l_run;
+                const float inv = nkv > 0 ? 1.f / l_run : 0.f;
                 const uint32_t stage = sQ + g * kTileBytes + r * 128;
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
                     uint32_t acc[32];
-                    tmem_ld32(tO + cb * 32, acc);
-                    tmem_wait_ld();
+                    if (nkv > 0) {
+                        tmem_ld32(tO + cb * 32, acc);
+                        tmem_wait_ld();
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[i] = 0u;       // no key: nothing was accumulated
+                    }
                     const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -273,7 +283,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (err == 0 && (warp & 3) == 0 && lane == 0) {
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_store_3d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, bh);
+                    tma_store_4d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, h_idx, b_idx);
                 tma_store_commit();
                 tma_store_wait_read();
             }
@@ -287,9 +297,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 mbar_expect_tx(bar_q(g), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_load_3d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM, bh);
+                    tma_load_4d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM,
+                                h_idx, b_idx);
             };
-            load_q(0);
+            if (nkv > 0) load_q(0);      // without keys the Q buffers only stage the zero output
             // ring items: 2j = K tile j, 2j+1 = V tile j
             for (int item = 0; item < 2 * nkv; ++item) {
                 if (item == 1 && ntiles > 1) load_q(1);
@@ -300,7 +311,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 mbar_expect_tx(bar_kv_full(slot), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_load_3d(dst + cx * kBoxBytes, tm, bar_kv_full(slot), cx * 64, (item >> 1) * kBlockN, bh);
+                    tma_load_4d(dst + cx * kBoxBytes, tm, bar_kv_full(slot), cx * 64, (item >> 1) * kBlockN, h_idx, b_idx);
             }
         } else if (warp == kMmaWarp && lane == 0) {
             // =============================================================== MMA issuer
@@ -338,6 +349,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 return mbar_wait(bar_kv_full(item % kStages), (item / kStages) & 1);
             };
             do {
+                if (nkv == 0) break;
                 if (!mbar_wait(bar_q(0), 0)) { err = kErrWaitQ; break; }
                 if (!wait_item(0)) { err = kErrWaitKV; break; }
                 tc_fence_after();
@@ -401,16 +413,21 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [BH, N, D] bf16, D innermost; box = 64 columns x 128 rows x 1, 128-byte swizzle, zero fill.
-int make_tmap(CUtensorMap *m, const void *base, int BH, int N, int D)
+// (D, N, H, B) bf16 view of a [B,H,N,D] (head_major) or [B,N,H,D] tensor, D innermost;
+// box = 64 columns x 128 rows x 1 x 1, 128-byte swizzle, zero fill: a tile never reaches
+// into the next head or sequence, and rows past N read as zero / are not written.
+int make_tmap(CUtensorMap *m, const void *base, int B, int H, int N, int D, bool head_major)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return dd::cuda_fail(cudaErrorSymbolNotFound, "cuTensorMapEncodeTiled entry point");
-    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
-    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)N * D * 2};
-    const cuuint32_t box[3] = {64, 128, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+    const cuuint64_t row = (cuuint64_t)D * 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {head_major ? row : row * H,           // between rows n
+                                   head_major ? row * N : row,           // between heads
+                                   row * N * H};                         // between sequences
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return dd::cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
@@ -436,17 +453,18 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
     return DD_OK;
 }
 
-int attention_impl(const void *q, const void *k, const void *v, void *out, int B, int H, int N, int D,
-                   float scale, void *stream)
+int attention_impl(const void *q, const void *k, const void *v, void *out, int B, int H, int Nq, int Nkv, int D,
+                   const int32_t *kv_len, int layout, float scale, void *stream)
 {
     if (!q || !k || !v || !out) return DD_ERR_INVALID_ARG;
-    if (B <= 0 || H <= 0 || N <= 0 || D <= 0) return DD_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || D <= 0) return DD_ERR_INVALID_ARG;
+    if (layout != DD_LAYOUT_BHND && layout != DD_LAYOUT_BNHD) return DD_ERR_INVALID_ARG;
     if (!isfinite(scale)) return DD_ERR_INVALID_ARG;
     if (scale < 0.f) return DD_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return DD_ERR_UNSUPPORTED;
     if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) != 0) return DD_ERR_UNSUPPORTED;
     const long BH = (long)B * H;
-    const int m_blocks = (N + kQTiles * kBlockM - 1) / (kQTiles * kBlockM);
+    const int m_blocks = (Nq + kQTiles * kBlockM - 1) / (kQTiles * kBlockM);
     if (BH * m_blocks >= (1L << 31) || BH >= (1L << 31)) return DD_ERR_UNSUPPORTED;
 
     dd::DeviceCtx *ctx = dd::current_ctx();
@@ -455,17 +473,18 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
         DD_CUDA_TRY(cudaMalloc(&ctx->attn_status, 256));
         DD_CUDA_TRY(cudaMemset(ctx->attn_status, 0, 256));
     }
+    const bool head_major = layout == DD_LAYOUT_BHND;
     CUtensorMap tq, tk, tv, to;
     int rc;
-    if ((rc = make_tmap(&tq, q, (int)BH, N, D)) != DD_OK) return rc;
-    if ((rc = make_tmap(&tk, k, (int)BH, N, D)) != DD_OK) return rc;
-    if ((rc = make_tmap(&tv, v, (int)BH, N, D)) != DD_OK) return rc;
-    if ((rc = make_tmap(&to, out, (int)BH, N, D)) != DD_OK) return rc;
+    if ((rc = make_tmap(&tq, q, B, H, Nq, D, head_major)) != DD_OK) return rc;
+    if ((rc = make_tmap(&tk, k, B, H, Nkv, D, head_major)) != DD_OK) return rc;
+    if ((rc = make_tmap(&tv, v, B, H, Nkv, D, head_major)) != DD_OK) return rc;
+    if ((rc = make_tmap(&to, out, B, H, Nq, D, head_major)) != DD_OK) return rc;
 
     AttnParams p;
-    p.out = (__nv_bfloat16 *)out;
-    p.BH = (int)BH; p.N = N; p.D = D;
+    p.BH = (int)BH; p.H = H; p.Nq = Nq; p.Nkv = Nkv; p.D = D;
     p.m_blocks = m_blocks;
+    p.kv_len = kv_len;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->attn_status;
     cudaStream_t s = (cudaStream_t)stream;
@@ -477,5 +496,12 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
 extern "C" int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
                                   int B, int H, int N, int D, float scale, void *stream)
 {
-    return attention_impl(q, k, v, out, B, H, N, D, scale, stream);
+    return attention_impl(q, k, v, out, B, H, N, N, D, nullptr, DD_LAYOUT_BHND, scale, stream);
+}
+
+extern "C" int dd_block_attention(const void *q, const void *k, const void *v, void *out,
+                                  int B, int H, int Nq, int Nkv, int D,
+                                  const int32_t *kv_len, int layout, float scale, void *stream)
+{
+    return attention_impl(q, k, v, out, B, H, Nq, Nkv, D, kv_len, layout, scale, stream);
 }

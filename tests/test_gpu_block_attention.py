@@ -1,0 +1,112 @@
+"""dd_block_attention on the GPU against the fp64 CPU oracle, through the C ABI:
+a block of queries over stored keys, ragged key counts, both memory layouts."""
+import numpy as np
+import pytest
+
+from paper_2604_05250_b200 import synth
+from tests._parity import bf16_tensor_to_f64, check_attention, to_torch_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dd():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2604_05250_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def block_inputs(B, H, Nq, Nkv, D, seed, planted=False):
+    if planted:
+        # queries and keys must share the planted subspace: one draw, the first Nq query rows
+        assert Nq <= Nkv
+        q, k, v = synth.attention_inputs(B, H, Nkv, D, seed, planted=True)
+        return np.ascontiguousarray(q[:, :, :Nq]), k, v
+    q, _, _ = synth.attention_inputs(B, H, Nq, D, seed)
+    _, k, v = synth.attention_inputs(B, H, Nkv, D, seed + 1)
+    return q, k, v
+
+
+def run_gpu(dd, q, k, v, scale, kv_len=None, layout="bhnd"):
+    import torch
+    tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
+    tl = None if kv_len is None else torch.from_numpy(np.asarray(kv_len, dtype=np.int32)).cuda()
+    out = dd.block_attention(tq, tk, tv, kv_len=tl, layout=layout, scale=scale)
+    torch.cuda.synchronize()
+    assert dd.attention_status() == 0
+    return bf16_tensor_to_f64(out)
+
+
+# query blocks shorter than, equal to and longer than one and two 128-row tiles; key counts
+# that end inside a tile, on a tile boundary and span several ring rounds
+@pytest.mark.parametrize("B,H,Nq,Nkv,D", [
+    (2, 3, 32, 1024, 128), (1, 4, 64, 1000, 128), (2, 2, 128, 130, 128), (1, 2, 200, 700, 64),
+    (1, 3, 300, 257, 128), (3, 2, 1, 1, 64), (1, 2, 256, 2048, 128),
+])
+def test_query_block_over_stored_keys(dd, oracle_mod, B, H, Nq, Nkv, D):
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 100 + Nq)
+    scale = D ** -0.5
+    got = run_gpu(dd, q, k, v, scale)
+    check_attention(got, oracle_mod.block_attention(q, k, v, scale))
+
+
+def test_ragged_key_counts_and_padding(dd, oracle_mod):
+    B, H, Nq, Nkv, D = 6, 2, 96, 640, 128
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 21)
+    kv_len = np.array([640, 1, 128, 129, 0, 511], dtype=np.int32)
+    # padding holds values that would dominate every row if it were read as keys
+    for b in range(B):
+        k[b, :, kv_len[b]:] = synth.f32_to_bf16_bits(np.float32(50.0))
+        v[b, :, kv_len[b]:] = synth.f32_to_bf16_bits(np.float32(1000.0))
+    got = run_gpu(dd, q, k, v, D ** -0.5, kv_len=kv_len)
+    ref = oracle_mod.block_attention(q, k, v, D ** -0.5, kv_len=kv_len)
+    check_attention(got, ref)
+    assert (got[4] == 0).all()                      # no valid key: zero output
+    # lengths outside [0, Nkv] are clamped
+    got2 = run_gpu(dd, q, k, v, D ** -0.5, kv_len=np.array([9999, 1, 128, 129, -5, 511], dtype=np.int32))
+    np.testing.assert_array_equal(got2, got)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_interleaved_head_layout(dd, oracle_mod, D):
+    B, H, Nq, Nkv = 2, 5, 160, 384
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 33)
+    kv_len = np.array([384, 200], dtype=np.int32)
+    tr = lambda a: np.ascontiguousarray(a.transpose(0, 2, 1, 3))
+    got = run_gpu(dd, tr(q), tr(k), tr(v), D ** -0.5, kv_len=kv_len, layout="bnhd")
+    ref = oracle_mod.block_attention(tr(q), tr(k), tr(v), D ** -0.5, kv_len=kv_len, layout="bnhd")
+    check_attention(got, ref)
+    # the same problem in the head-major layout gives the same bits
+    got_hm = run_gpu(dd, q, k, v, D ** -0.5, kv_len=kv_len, layout="bhnd")
+    np.testing.assert_array_equal(tr(got_hm), got)
+
+
+def test_square_case_is_the_bidirectional_kernel(dd):
+    import torch
+    q, k, v = synth.attention_inputs(1, 4, 333, 128, 5)
+    tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
+    a = dd.bidir_attention(tq, tk, tv)
+    b = dd.block_attention(tq, tk, tv)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_peaked_rows_with_planted_structure(dd, oracle_mod):
+    q, k, v = block_inputs(1, 2, 128, 1536, 128, 44, planted=True)
+    got = run_gpu(dd, q, k, v, 128 ** -0.5, kv_len=np.array([1500], dtype=np.int32))
+    check_attention(got, oracle_mod.block_attention(q, k, v, 128 ** -0.5, kv_len=np.array([1500], dtype=np.int32)))
+
+
+def test_argument_errors(dd):
+    import torch
+    q = torch.zeros(1, 2, 16, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(1, 2, 32, 128, dtype=torch.bfloat16, device="cuda")
+    L = dd.lib()
+    p = lambda t: t.data_ptr()
+    assert L.dd_block_attention(p(q), p(k), p(k), p(q), 1, 2, 16, 32, 128, None, 7, 0.1, None) == dd.DD_ERR_INVALID_ARG
+    assert L.dd_block_attention(p(q), p(k), p(k), p(q), 1, 2, 0, 32, 128, None, 0, 0.1, None) == dd.DD_ERR_INVALID_ARG
+    assert L.dd_block_attention(p(q), p(k), p(k), p(q), 1, 2, 16, 32, 96, None, 0, 0.1, None) == dd.DD_ERR_UNSUPPORTED
+    assert L.dd_block_attention(None, p(k), p(k), p(q), 1, 2, 16, 32, 128, None, 0, 0.1, None) == dd.DD_ERR_INVALID_ARG
