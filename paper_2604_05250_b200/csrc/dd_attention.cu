@@ -7,9 +7,9 @@
 // the keys in tiles of 128.  The CTA is warp-specialised:
 //   warps 0-3   softmax of query tile 0 (thread = query row = TMEM lane)
 //   warps 4-7   softmax of query tile 1
-//   warp  8     one thread feeds a ring of K/V tiles by TMA (4-D tensor maps over
-//               (D, N, H, B) with the strides of the layout, 128-byte swizzle; rows
-//               past N read as zero)
+//   warp  8     one thread feeds a ring of K/V tiles by TMA (tensor maps over
+//               (D, N, B*H) or, heads interleaved, (D, N, H, B); 128-byte swizzle;
+//               rows past N read as zero)
 //   warp  9     one thread issues every tcgen05 MMA
 // S_g = Q_g K^T goes to tensor memory; the softmax thread reads its row, keeps the
 // running maximum and sum in fp32 (online softmax in base 2, scale*log2e folded
@@ -48,6 +48,7 @@ struct AttnParams {
     int BH, H, Nq, Nkv, D;
     int m_blocks;              // CTAs per (batch, head) = ceil(Nq / 256)
     const int *kv_len;         // [B] keys of each sequence that exist (clamped to 0..Nkv), or null: Nkv
+    int head_major;            // 1: [B,H,N,D], tensor maps are 3-D over (D, N, B*H); 0: [B,N,H,D], 4-D maps (D, N, H, B)
     float scale_log2;          // scale * log2(e)
     unsigned int *status;
 };
@@ -127,7 +128,9 @@ __device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int 
     return sum2.x + sum2.y;
 }
 
-template <int D>
+// kBlock = false: the square, head-major, unpadded case of dd_bidir_attention with nothing of the
+// general case compiled in.
+template <int D, bool kBlock>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -153,8 +156,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int bh = blockIdx.x / p.m_blocks;
     const int mb = blockIdx.x - bh * p.m_blocks;
     const int row0 = mb * (kQTiles * kBlockM);
-    const int b_idx = bh / p.H, h_idx = bh - b_idx * p.H;
-    const int keys = p.kv_len ? min(max(p.kv_len[b_idx], 0), p.Nkv) : p.Nkv;   // keys that exist
+    const int b_idx = kBlock ? bh / p.H : 0, h_idx = kBlock ? bh - b_idx * p.H : 0;
+    const bool hm = !kBlock || p.head_major != 0;
+    // one tile of 128 rows x 64 columns of head (b_idx, h_idx), rows from n0
+    auto load_box = [&](uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int n0) {
+        if (hm) tma_load_3d(dst, tm, bar, c0, n0, bh);
+        else tma_load_4d(dst, tm, bar, c0, n0, h_idx, b_idx);
+    };
+    const int keys = (kBlock && p.kv_len) ? min(max(p.kv_len[b_idx], 0), p.Nkv) : p.Nkv;   // keys that exist
     const int nkv = (keys + kBlockN - 1) / kBlockN;       // 0: the sequence has no key, the output is zero
     const int ntiles = (p.Nq - row0 > kBlockM) ? 2 : 1;   // query tiles of this CTA that hold rows
     constexpr int kBoxes = D / 64;                 // 64-column (128-byte) boxes per tile row
@@ -241,19 +250,19 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 tc_fence_before();
                 mbar_arrive(bar_p_full(g));
             }
-            if (err == 0 && nkv > 0 && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
+            if (err == 0 && (!kBlock || nkv > 0) && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
             if (err == 0) {
                 // ---- epilogue: O / l -> bf16 -> this tile's Q buffer (every MMA that read it has
                 // completed), in the swizzled layout of the tensor map, -> global by TMA (rows past N
                 // are clipped by the map)
                 tc_fence_after();
                 const int r = (warp & 3) * 32 + lane;                 // row within the tile
-                const float inv = nkv > 0 ? 1.f / l_run : 0.f;
+                const float inv = (!kBlock || nkv > 0) ? 1.f / l_run : 0.f;
                 const uint32_t stage = sQ + g * kTileBytes + r * 128;
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
                     uint32_t acc[32];
-                    if (nkv > 0) {
+                    if (!kBlock || nkv > 0) {
                         tmem_ld32(tO + cb * 32, acc);
                         tmem_wait_ld();
                     } else {
@@ -283,7 +292,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (err == 0 && (warp & 3) == 0 && lane == 0) {
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_store_4d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, h_idx, b_idx);
+                    if (hm) tma_store_3d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, bh);
+                    else tma_store_4d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, h_idx, b_idx);
                 tma_store_commit();
                 tma_store_wait_read();
             }
@@ -297,10 +307,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 mbar_expect_tx(bar_q(g), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_load_4d(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM,
-                                h_idx, b_idx);
+                    load_box(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM);
             };
-            if (nkv > 0) load_q(0);      // without keys the Q buffers only stage the zero output
+            if (!kBlock || nkv > 0) load_q(0);      // without keys the Q buffers only stage the zero output
             // ring items: 2j = K tile j, 2j+1 = V tile j
             for (int item = 0; item < 2 * nkv; ++item) {
                 if (item == 1 && ntiles > 1) load_q(1);
@@ -311,7 +320,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 mbar_expect_tx(bar_kv_full(slot), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    tma_load_4d(dst + cx * kBoxBytes, tm, bar_kv_full(slot), cx * 64, (item >> 1) * kBlockN, h_idx, b_idx);
+                    load_box(dst + cx * kBoxBytes, tm, bar_kv_full(slot), cx * 64, (item >> 1) * kBlockN);
             }
         } else if (warp == kMmaWarp && lane == 0) {
             // =============================================================== MMA issuer
@@ -349,7 +358,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 return mbar_wait(bar_kv_full(item % kStages), (item / kStages) & 1);
             };
             do {
-                if (nkv == 0) break;
+                if (kBlock && nkv == 0) break;
                 if (!mbar_wait(bar_q(0), 0)) { err = kErrWaitQ; break; }
                 if (!wait_item(0)) { err = kErrWaitKV; break; }
                 tc_fence_after();
@@ -413,28 +422,36 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// (D, N, H, B) bf16 view of a [B,H,N,D] (head_major) or [B,N,H,D] tensor, D innermost;
-// box = 64 columns x 128 rows x 1 x 1, 128-byte swizzle, zero fill: a tile never reaches
-// into the next head or sequence, and rows past N read as zero / are not written.
+// bf16 view of a [B,H,N,D] tensor as (D, N, B*H) (head_major: batch and head merge into one
+// dimension) or of a [B,N,H,D] tensor as (D, N, H, B); box = 64 columns x 128 rows x 1 (x 1),
+// 128-byte swizzle, zero fill: a tile never reaches into the next head or sequence, and rows
+// past N read as zero / are not written.
 int make_tmap(CUtensorMap *m, const void *base, int B, int H, int N, int D, bool head_major)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return dd::cuda_fail(cudaErrorSymbolNotFound, "cuTensorMapEncodeTiled entry point");
     const cuuint64_t row = (cuuint64_t)D * 2;
-    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {head_major ? row : row * H,           // between rows n
-                                   head_major ? row * N : row,           // between heads
-                                   row * N * H};                         // between sequences
     const cuuint32_t box[4] = {64, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r;
+    if (head_major) {
+        const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)B * H};
+        const cuuint64_t strides[2] = {row, row * N};
+        r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+        const cuuint64_t strides[3] = {row * H, row, row * N * H};      // between rows, heads, sequences
+        r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) return dd::cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     return DD_OK;
 }
 
-template <int D>
+template <int D, bool kBlock>
 int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
            const AttnParams &p, cudaStream_t s)
 {
@@ -443,11 +460,11 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
     DD_CUDA_TRY(cudaGetDevice(&dev));
     const int smem = Smem<D>::kTotal + 1024;
     if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        DD_CUDA_TRY(cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        DD_CUDA_TRY(cudaFuncSetAttribute(attention_kernel<D, kBlock>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr_done[dev] = true;
     }
     const long grid = (long)p.BH * p.m_blocks;
-    attention_kernel<D><<<(unsigned)grid, kThreads, smem, s>>>(tq, tk, tv, to, p);
+    attention_kernel<D, kBlock><<<(unsigned)grid, kThreads, smem, s>>>(tq, tk, tv, to, p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
     return DD_OK;
@@ -485,10 +502,13 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     p.BH = (int)BH; p.H = H; p.Nq = Nq; p.Nkv = Nkv; p.D = D;
     p.m_blocks = m_blocks;
     p.kv_len = kv_len;
+    p.head_major = head_major ? 1 : 0;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->attn_status;
     cudaStream_t s = (cudaStream_t)stream;
-    return D == 64 ? launch<64>(tq, tk, tv, to, p, s) : launch<128>(tq, tk, tv, to, p, s);
+    const bool general = kv_len != nullptr || !head_major || Nq != Nkv;
+    if (general) return D == 64 ? launch<64, true>(tq, tk, tv, to, p, s) : launch<128, true>(tq, tk, tv, to, p, s);
+    return D == 64 ? launch<64, false>(tq, tk, tv, to, p, s) : launch<128, false>(tq, tk, tv, to, p, s);
 }
 
 }  // namespace

@@ -84,14 +84,17 @@ def test_interleaved_head_layout(dd, oracle_mod, D):
     np.testing.assert_array_equal(tr(got_hm), got)
 
 
-def test_square_case_is_the_bidirectional_kernel(dd):
+def test_square_case_equals_bidirectional_attention(dd):
+    """Nq = Nkv with every key valid: the general instantiation (forced by passing kv_len)
+    gives the same bits as dd_bidir_attention."""
     import torch
-    q, k, v = synth.attention_inputs(1, 4, 333, 128, 5)
+    q, k, v = synth.attention_inputs(2, 4, 333, 128, 5)
     tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
     a = dd.bidir_attention(tq, tk, tv)
     b = dd.block_attention(tq, tk, tv)
+    c = dd.block_attention(tq, tk, tv, kv_len=torch.tensor([333, 400], dtype=torch.int32, device="cuda"))
     torch.cuda.synchronize()
-    assert torch.equal(a, b)
+    assert torch.equal(a, b) and torch.equal(a, c)
 
 
 def test_peaked_rows_with_planted_structure(dd, oracle_mod):
