@@ -166,6 +166,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int keys = (kBlock && p.kv_len) ? min(max(p.kv_len[b_idx], 0), p.Nkv) : p.Nkv;   // keys that exist
     const int nkv = (keys + kBlockN - 1) / kBlockN;       // 0: the sequence has no key, the output is zero
     const int ntiles = (p.Nq - row0 > kBlockM) ? 2 : 1;   // query tiles of this CTA that hold rows
+    // A CTA with a single query tile (a short query block) gives its key tiles to the two softmax
+    // groups in turn: both keep a copy of the query tile and an accumulator of their own, and the
+    // two partial results are combined at the end.  The tensor core then works for one group
+    // while the other computes its weights, as with two query tiles.
+    const bool split = kBlock && ntiles == 1 && nkv >= 2;
+    const int groups = split ? 2 : ntiles;                // softmax groups at work
     constexpr int kBoxes = D / 64;                 // 64-column (128-byte) boxes per tile row
     constexpr uint32_t kBoxBytes = 128 * 128;      // 128 rows x 128 bytes
     constexpr uint32_t kColS = 0, kColO = 256;
@@ -203,9 +209,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         float m_ref = -INFINITY, l_run = 0.f;
         unsigned err = 0;
 
-        if (g < ntiles) {
-            for (int j = 0; j < nkv; ++j) {
-                if (!mbar_wait(bar_s_full(g), j & 1)) { err = kErrWaitS; break; }
+        // key tiles of this group: j_first, j_first + j_step, ...
+        const int j_first = split ? g : 0, j_step = split ? 2 : 1;
+        const int my_tiles = nkv > j_first ? (nkv - j_first + j_step - 1) / j_step : 0;
+        if (g < groups) {
+            for (int i = 0; i < my_tiles; ++i) {
+                const int j = j_first + i * j_step;
+                if (!mbar_wait(bar_s_full(g), i & 1)) { err = kErrWaitS; break; }
                 tc_fence_after();
                 float s[kBlockN];
 #pragma unroll
@@ -219,7 +229,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 // weighted against the reference point they inherit, in one pass, and only a row
                 // whose maximum turns out to have grown past it by more than the allowed step moves
                 // the reference point, rescales O and weights the tile again.
-                if (j == 0) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
+                if (i == 0) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
                 float mx;
                 float sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
                                    : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
@@ -230,7 +240,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     m_ref = m_new;
                     l_run *= alpha;
                     // O_g holds the sum over tiles < j once the previous P V has completed
-                    if (!mbar_wait(bar_o_full(g), (j - 1) & 1)) { err = kErrWaitO; break; }
+                    if (!mbar_wait(bar_o_full(g), (i - 1) & 1)) { err = kErrWaitO; break; }
                     tc_fence_after();
 #pragma unroll
                     for (int cb = 0; cb < D / 32; ++cb) {
@@ -250,14 +260,39 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 tc_fence_before();
                 mbar_arrive(bar_p_full(g));
             }
-            if (err == 0 && (!kBlock || nkv > 0) && !mbar_wait(bar_o_full(g), (nkv - 1) & 1)) err = kErrWaitO;
-            if (err == 0) {
+            if (err == 0 && (!kBlock || nkv > 0) && !mbar_wait(bar_o_full(g), (my_tiles - 1) & 1)) err = kErrWaitO;
+            // ---- split keys: group 1 hands its reference point and row sum to group 0 (through its
+            // own Q buffer, which no MMA reads any more) and is done; group 0 adds group 1's
+            // accumulator, read from tensor memory, to its own.  Every thread of both groups takes
+            // part in the hand-over, also after an expired wait.
+            float scale_own = 1.f, scale_other = 0.f;
+            float2 *hand_over = reinterpret_cast<float2 *>(smem_gen + Smem<D>::kQ + kTileBytes);
+            if (kBlock && split) {
+                const int r = (warp & 3) * 32 + lane;
+                if (g == 1) {
+                    hand_over[r] = make_float2(m_ref, l_run);
+                    __threadfence_block();
+                    named_bar_arrive(3, 2 * kBlockM);
+                } else {
+                    named_bar_sync(3, 2 * kBlockM);
+                    const float2 other = hand_over[r];
+                    if (err == 0 && !mbar_wait(bar_o_full(1), ((nkv / 2) - 1) & 1)) err = kErrWaitO;
+                    const float m_all = fmaxf(m_ref, other.x);
+                    scale_own = ex2(m_ref - m_all);
+                    scale_other = ex2(other.x - m_all);
+                    l_run = l_run * scale_own + other.y * scale_other;
+                }
+            }
+            if (err != 0) report(p.status, err);
+            const bool stores = !(kBlock && split && g == 1);
+            if (stores && err == 0) {
                 // ---- epilogue: O / l -> bf16 -> this tile's Q buffer (every MMA that read it has
                 // completed), in the swizzled layout of the tensor map, -> global by TMA (rows past N
                 // are clipped by the map)
                 tc_fence_after();
                 const int r = (warp & 3) * 32 + lane;                 // row within the tile
                 const float inv = (!kBlock || nkv > 0) ? 1.f / l_run : 0.f;
+                const float w_own = scale_own * inv, w_other = scale_other * inv;
                 const uint32_t stage = sQ + g * kTileBytes + r * 128;
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
@@ -265,6 +300,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     if (!kBlock || nkv > 0) {
                         tmem_ld32(tO + cb * 32, acc);
                         tmem_wait_ld();
+                        if (kBlock && split) {
+                            uint32_t acc1[32];
+                            tmem_ld32(tO + D + cb * 32, acc1);          // group 1's accumulator, same rows
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                acc[i] = __float_as_uint(__uint_as_float(acc[i]) * w_own + __uint_as_float(acc1[i]) * w_other);
+                        }
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) acc[i] = 0u;       // no key: nothing was accumulated
@@ -275,8 +318,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         uint32_t w[4];
 #pragma unroll
                         for (int h = 0; h < 4; ++h) {
-                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * inv,
-                                                                     __uint_as_float(acc[i + 2 * h + 1]) * inv);
+                            const float f = (kBlock && split) ? 1.f : inv;      // split: already weighted
+                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * f,
+                                                                     __uint_as_float(acc[i + 2 * h + 1]) * f);
                             w[h] = *reinterpret_cast<uint32_t *>(&v);
                         }
                         const int chunk = (cb % 2) * 4 + i / 8;         // 16-byte chunk of the 128-byte row
@@ -284,12 +328,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     }
                 }
                 fence_proxy_async_smem();
-            } else {
-                report(p.status, err);
             }
             // every thread of the warpgroup comes here, also after an expired wait
             named_bar_sync(1 + g, kBlockM);
-            if (err == 0 && (warp & 3) == 0 && lane == 0) {
+            if (stores && err == 0 && (warp & 3) == 0 && lane == 0) {
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
                     if (hm) tma_store_3d(&tm_o, sQ + g * kTileBytes + cx * kBoxBytes, cx * 64, row0 + g * kBlockM, bh);
@@ -303,16 +345,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (warp == kLoadWarp && lane == 0) {
             // =============================================================== TMA producer
             // what the first MMA needs comes first: Q tile 0, K tile 0, then Q tile 1
+            // buffer g takes query tile g, or, with split keys, a second copy of tile 0
             auto load_q = [&](int g) {
                 mbar_expect_tx(bar_q(g), kTileBytes);
 #pragma unroll
                 for (int cx = 0; cx < kBoxes; ++cx)
-                    load_box(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64, row0 + g * kBlockM);
+                    load_box(sQ + g * kTileBytes + cx * kBoxBytes, &tm_q, bar_q(g), cx * 64,
+                             row0 + (split ? 0 : g * kBlockM));
             };
             if (!kBlock || nkv > 0) load_q(0);      // without keys the Q buffers only stage the zero output
             // ring items: 2j = K tile j, 2j+1 = V tile j
             for (int item = 0; item < 2 * nkv; ++item) {
-                if (item == 1 && ntiles > 1) load_q(1);
+                if (item == 1 && groups > 1) load_q(1);
                 const int slot = item % kStages, use = item / kStages;
                 if (use > 0 && !mbar_wait(bar_kv_empty(slot), (use - 1) & 1)) { report(p.status, kErrWaitSlot); break; }
                 const uint32_t dst = sRing + slot * kTileBytes;
@@ -357,6 +401,34 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             auto wait_item = [&](int item) {
                 return mbar_wait(bar_kv_full(item % kStages), (item / kStages) & 1);
             };
+            // Split keys: key tile t belongs to group t & 1.  S_0(0), S_1(1), then per tile t:
+            // O_g (+)= P_g V_t, S_g(t + 2).  Every ring item is read by one group only.
+            if (kBlock && split) {
+                do {
+                    for (int g = 0; g < 2; ++g) {
+                        if (!mbar_wait(bar_q(g), 0)) { err = kErrWaitQ; break; }
+                        if (!wait_item(2 * g)) { err = kErrWaitKV; break; }
+                        tc_fence_after();
+                        issue_s(g, (2 * g) % kStages);
+                        mma_commit(bar_kv_empty((2 * g) % kStages));
+                    }
+                    for (int t = 0; t < nkv && err == 0; ++t) {
+                        const int g = t & 1, i = t >> 1;
+                        const int item_v = 2 * t + 1, item_k = 2 * (t + 2);
+                        if (!wait_item(item_v)) { err = kErrWaitKV; break; }
+                        if (!mbar_wait(bar_p_full(g), i & 1)) { err = kErrWaitP; break; }
+                        tc_fence_after();
+                        issue_o(g, item_v % kStages, i == 0);
+                        mma_commit(bar_kv_empty(item_v % kStages));
+                        if (t + 2 < nkv) {
+                            if (!wait_item(item_k)) { err = kErrWaitKV; break; }
+                            tc_fence_after();
+                            issue_s(g, item_k % kStages);
+                            mma_commit(bar_kv_empty(item_k % kStages));
+                        }
+                    }
+                } while (false);
+            } else
             do {
                 if (kBlock && nkv == 0) break;
                 if (!mbar_wait(bar_q(0), 0)) { err = kErrWaitQ; break; }

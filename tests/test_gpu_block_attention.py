@@ -86,15 +86,24 @@ def test_interleaved_head_layout(dd, oracle_mod, D):
 
 def test_square_case_equals_bidirectional_attention(dd):
     """Nq = Nkv with every key valid: the general instantiation (forced by passing kv_len)
-    gives the same bits as dd_bidir_attention."""
+    gives the same bits as dd_bidir_attention where every CTA holds two query tiles; a CTA
+    with a single query tile splits its keys between the softmax groups, which changes the
+    order of the sums but not the result beyond rounding."""
     import torch
-    q, k, v = synth.attention_inputs(2, 4, 333, 128, 5)
-    tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
-    a = dd.bidir_attention(tq, tk, tv)
-    b = dd.block_attention(tq, tk, tv)
-    c = dd.block_attention(tq, tk, tv, kv_len=torch.tensor([333, 400], dtype=torch.int32, device="cuda"))
-    torch.cuda.synchronize()
-    assert torch.equal(a, b) and torch.equal(a, c)
+    for N, exact in ((512, True), (333, False)):
+        q, k, v = synth.attention_inputs(2, 4, N, 128, 5)
+        tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
+        a = dd.bidir_attention(tq, tk, tv)
+        b = dd.block_attention(tq, tk, tv)
+        c = dd.block_attention(tq, tk, tv, kv_len=torch.tensor([N, N + 67], dtype=torch.int32, device="cuda"))
+        torch.cuda.synchronize()
+        assert dd.attention_status() == 0
+        assert torch.equal(a, b)
+        if exact:
+            assert torch.equal(a, c)
+        else:
+            assert torch.equal(a[:, :, :256], c[:, :, :256])
+            assert (a.float() - c.float()).abs().max().item() <= 4e-3
 
 
 def test_peaked_rows_with_planted_structure(dd, oracle_mod):
