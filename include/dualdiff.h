@@ -108,6 +108,28 @@ int dd_verify(const void *drafter_logits, const void *verifier_logits,
               int32_t *out_tokens, uint8_t *out_mask, float *out_score,
               int B, int P, int V, void *stream);
 
+/*
+ * Unmask(p, x): one confidence-based unmasking step of a masked diffusion
+ * model, the operation the drafter applies K times per cycle (Algorithm 1,
+ * drafting phase; Section 2.1; Section 2.3 for the threshold rule versus a
+ * fixed number per step).  For every position with mask_flags == 1 (currently
+ * [MASK]): a_i = argmax_x logits[b,i,x] (lowest index), c_i = softmax(logits[b,i,:])(a_i).
+ * The position is unmasked iff c_i >= tau, or it is one of the k most confident
+ * masked positions of its sequence (ties to the lower i).  tau = +infinity
+ * unmasks exactly min(k, masked) positions per sequence; k = 1 guarantees
+ * progress under a threshold; k = 0 leaves the threshold alone.
+ *   out_tokens[b,i] = a_i if unmasked, else tokens[b,i] (the caller's [MASK] id)
+ *   out_mask[b,i]   = 1 if the position stays masked, else 0
+ *   out_conf[b,i]   = c_i (nullable)
+ * Positions with mask_flags == 0 pass through (out_tokens = tokens, out_mask = 0,
+ * out_conf = 0) and their logits are never read.  Shapes, supported sizes,
+ * scratch and errors as for dd_verify, whose confidence rule (Eq. 7) this is,
+ * applied to one logits tensor: the same kernel launch.
+ */
+int dd_unmask(const void *logits, const int32_t *tokens, const uint8_t *mask_flags,
+              float tau, int k, int32_t *out_tokens, uint8_t *out_mask, float *out_conf,
+              int B, int P, int V, void *stream);
+
 /* `layout` argument of dd_block_attention. */
 enum {
     DD_LAYOUT_BHND = 0, /* q, out [B,H,Nq,D]; k, v [B,H,Nkv,D]                     */

@@ -55,6 +55,8 @@ def _load():
         lib.dd_oracle_verify.argtypes = [vp, vp, vp, vp, i32, f64, i32, u64,
                                          vp, vp, vp, vp, i32, i32, i32]
         lib.dd_oracle_verify.restype = i32
+        lib.dd_oracle_unmask.argtypes = [vp, vp, vp, f64, i32, vp, vp, vp, vp, i32, i32, i32]
+        lib.dd_oracle_unmask.restype = None
         lib.dd_oracle_threads.argtypes = []
         lib.dd_oracle_threads.restype = i32
         _lib = lib
@@ -183,3 +185,22 @@ def verify(drafter, verifier, tokens, flags, mode, tau, k, seed):
     if rc != 0:
         raise ValueError(f"dd_oracle_verify rejected its arguments (rc={rc})")
     return dict(out_tokens=out_tokens, out_mask=out_mask, out_score=out_score, exempt=exempt)
+
+
+def unmask(logits, tokens, flags, tau, k):
+    """One confidence-based unmasking step (Algorithm 1's Unmask).  Returns a dict with
+    out_tokens int32 [B,P], out_mask uint8 [B,P] (1 = still masked), out_conf float64 [B,P],
+    exempt uint8 [B,P]."""
+    logits = _u16(logits)
+    B, P, V = logits.shape
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    flags = np.ascontiguousarray(flags, dtype=np.uint8)
+    assert tokens.shape == (B, P) and flags.shape == (B, P)
+    out_tokens = np.empty((B, P), dtype=np.int32)
+    out_mask = np.empty((B, P), dtype=np.uint8)
+    out_conf = np.empty((B, P), dtype=np.float64)
+    exempt = np.empty((B, P), dtype=np.uint8)
+    tau32 = float(np.float32(tau))        # the CUDA library receives tau as a C float
+    _load().dd_oracle_unmask(_ptr(logits), _ptr(tokens), _ptr(flags), tau32, int(k),
+                             _ptr(out_tokens), _ptr(out_mask), _ptr(out_conf), _ptr(exempt), B, P, V)
+    return dict(out_tokens=out_tokens, out_mask=out_mask, out_conf=out_conf, exempt=exempt)

@@ -33,6 +33,13 @@
  *                              that the paper does not fix: PARITY UNPINNED
  *                              for those two (checked only against a brute
  *                              force restatement of the same reading).
+ *   dd_oracle_unmask           pinned for the threshold rule and the fixed
+ *                              number per step (hand-built cases, scipy
+ *                              softmax + numpy argsort on random inputs,
+ *                              monotonicity in tau); which of the two rules
+ *                              a caller combines, and ties to the lower
+ *                              position, are readings: PARITY UNPINNED for
+ *                              the tie order.
  */
 #include <math.h>
 #include <stdint.h>
@@ -404,6 +411,87 @@ int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
     free(members); free(rel); free(rank);
     free(amax); free(conf); free(kl);
     return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Unmask(p, x): one confidence-based unmasking step of a masked diffusion
+ * model (Algorithm 1, drafting phase; Section 2.1: "a subset of
+ * high-confidence tokens are unmasked"; Section 2.3: all tokens above a
+ * confidence threshold, rather than a fixed number per step).
+ *
+ * For every masked position i (flags = 1): p_i = softmax(logits_i),
+ * a_i = argmax (lowest index), c_i = p_i(a_i).  Position i is unmasked iff
+ * c_i >= tau, or it is one of the k most confident masked positions of its
+ * sequence (ties to the lower position).  tau = +inf gives "a fixed number k
+ * per step"; k = 1 guarantees progress under a threshold.
+ *
+ * out_tokens = a_i where unmasked, tokens[i] otherwise; out_mask = 1 where the
+ * position stays masked; out_conf = c_i (0 at positions that were not masked);
+ * exempt (nullable) = 1 where the decision lies within 1e-5 of the threshold
+ * or of the k-th / (k+1)-th confidence.                                     */
+typedef struct { double c; int pos; } conf_pos;
+
+static int more_confident_first(const void *x, const void *y)
+{
+    const conf_pos *a = (const conf_pos *)x, *b = (const conf_pos *)y;
+    if (a->c > b->c) return -1;
+    if (a->c < b->c) return 1;
+    return a->pos < b->pos ? -1 : (a->pos > b->pos ? 1 : 0);
+}
+
+void dd_oracle_unmask(const uint16_t *logits, const int32_t *tokens, const uint8_t *flags,
+                      double tau, int k,
+                      int32_t *out_tokens, uint8_t *out_mask, double *out_conf, uint8_t *exempt,
+                      int B, int P, int V)
+{
+    const long BP = (long)B * P;
+    int32_t *best = (int32_t *)malloc(sizeof(int32_t) * (size_t)BP);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long t = 0; t < BP; ++t) {
+        best[t] = 0;
+        out_conf[t] = 0.0;
+        if (!flags[t]) continue;
+        const uint16_t *row = logits + (size_t)t * V;
+        double top = -INFINITY;
+        int where = 0;
+        for (int x = 0; x < V; ++x) {
+            const double l = bf16_to_f64(row[x]);
+            if (l > top) { top = l; where = x; }
+        }
+        double denom = 0.0;
+        for (int x = 0; x < V; ++x) denom += exp(bf16_to_f64(row[x]) - top);
+        best[t] = where;
+        out_conf[t] = 1.0 / denom;           /* exp(top - top) / denom */
+    }
+    conf_pos *order = (conf_pos *)malloc(sizeof(conf_pos) * (size_t)P);
+    for (int b = 0; b < B; ++b) {
+        const long base = (long)b * P;
+        int n = 0;
+        for (int i = 0; i < P; ++i) {
+            out_tokens[base + i] = tokens[base + i];
+            out_mask[base + i] = 0;
+            if (exempt) exempt[base + i] = 0;
+            if (flags[base + i]) { order[n].c = out_conf[base + i]; order[n].pos = i; ++n; }
+        }
+        qsort(order, (size_t)n, sizeof(conf_pos), more_confident_first);
+        for (int r = 0; r < n; ++r) {
+            const long t = base + order[r].pos;
+            const int above = order[r].c >= tau;
+            const int unmask = above || r < k;
+            out_mask[t] = (uint8_t)!unmask;
+            if (unmask) out_tokens[t] = best[t];
+            if (exempt) {
+                int near = fabs(order[r].c - tau) <= EXEMPT_BAND;
+                if (!above && k > 0 && k < n) {      /* the top-k boundary decides */
+                    if (fabs(order[r].c - order[k - 1].c) <= EXEMPT_BAND) near = 1;
+                    if (fabs(order[r].c - order[k].c) <= EXEMPT_BAND) near = 1;
+                }
+                exempt[t] = (uint8_t)near;
+            }
+        }
+    }
+    free(order);
+    free(best);
 }
 
 /* Number of OpenMP threads a parallel region will use (reported by the bench). */

@@ -21,7 +21,7 @@ DD_LAYOUT_BHND, DD_LAYOUT_BNHD = 0, 1
 
 # every symbol include/dualdiff.h declares
 EXPORTS = (
-    "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
+    "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_unmask", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
     "dd_status_string", "dd_last_cuda_error", "dd_version",
 )
@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.dd_verify.argtypes = ver
         L.dd_verify_host.argtypes = ver
         L.dd_verify_static.argtypes = ver
+        L.dd_unmask.argtypes = [vp, vp, vp, f32, i32, vp, vp, vp, i32, i32, i32, vp]
+        L.dd_unmask.restype = i32
         L.dd_verify_static.restype = i32
         for name in ("dd_bidir_attention", "dd_bidir_attention_host", "dd_verify", "dd_verify_host",
                      "dd_attention_status", "dd_verify_status", "dd_release", "dd_version"):
@@ -188,6 +190,30 @@ def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, se
               int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
               _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, V, _stream_ptr(stream)))
     return out_tokens, out_mask, out_score
+
+
+def unmask(logits, tokens, mask_flags, tau, k, out_tokens=None, out_mask=None, out_conf=None, stream=None):
+    """dd_unmask: one confidence-based unmasking step on logits [B,P,V] (device tensors).
+
+    Returns (out_tokens int32 [B,P], out_mask uint8 [B,P] with 1 = still masked, out_conf float32 [B,P])."""
+    import torch
+    B, P, V = logits.shape
+    _require(logits, torch.bfloat16, (B, P, V), True, "logits")
+    _require(tokens, torch.int32, (B, P), True, "tokens")
+    _require(mask_flags, torch.uint8, (B, P), True, "mask_flags")
+    kw = dict(device=logits.device)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, P), dtype=torch.int32, **kw)
+    if out_mask is None:
+        out_mask = torch.empty((B, P), dtype=torch.uint8, **kw)
+    if out_conf is None:
+        out_conf = torch.empty((B, P), dtype=torch.float32, **kw)
+    _require(out_tokens, torch.int32, (B, P), True, "out_tokens")
+    _require(out_mask, torch.uint8, (B, P), True, "out_mask")
+    _require(out_conf, torch.float32, (B, P), True, "out_conf")
+    _check(lib().dd_unmask(_ptr(logits), _ptr(tokens), _ptr(mask_flags), float(tau), int(k),
+                           _ptr(out_tokens), _ptr(out_mask), _ptr(out_conf), B, P, V, _stream_ptr(stream)))
+    return out_tokens, out_mask, out_conf
 
 
 def attention_status() -> int:

@@ -366,6 +366,17 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     return launch(p, streaming, (cudaStream_t)stream);
 }
 
+// Unmask(p, x) of Algorithm 1's drafting phase: the confidence rule of dd_verify on one logits
+// tensor.  "Stays masked" is "fails the threshold and is not among the k most confident": the
+// CONF-mode decision with the roles of the outputs renamed, so it runs the same launch.
+extern "C" int dd_unmask(const void *logits, const int32_t *tokens, const uint8_t *mask_flags,
+                         float tau, int k, int32_t *out_tokens, uint8_t *out_mask, float *out_conf,
+                         int B, int P, int V, void *stream)
+{
+    return dd_verify(nullptr, logits, tokens, mask_flags, DD_MODE_CONF, tau, k, 0, out_tokens, out_mask, out_conf,
+                     B, P, V, stream);
+}
+
 extern "C" int dd_verify_status(void)
 {
     dd::DeviceCtx *ctx = dd::current_ctx();
