@@ -395,9 +395,11 @@ int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
             }
             /* Step 4: the k most reliable positions are kept whatever Step 3 said */
             const int in_topk = rank[a] < k;
+            /* the top-k rule decides a failing position; its place relative to the boundary is
+             * uncertain only if the reliability on the other side of the boundary is within the band */
             if (fail) {
-                if (!isnan(r_last_in) && fabs(rel[a] - r_last_in) <= EXEMPT_BAND) near = 1;
-                if (!isnan(r_first_out) && fabs(rel[a] - r_first_out) <= EXEMPT_BAND) near = 1;
+                if (in_topk && !isnan(r_first_out) && fabs(rel[a] - r_first_out) <= EXEMPT_BAND) near = 1;
+                if (!in_topk && !isnan(r_last_in) && fabs(rel[a] - r_last_in) <= EXEMPT_BAND) near = 1;
             }
             const int remask = fail && !in_topk;
             /* Step 5 */
@@ -427,8 +429,9 @@ int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
  *
  * out_tokens = a_i where unmasked, tokens[i] otherwise; out_mask = 1 where the
  * position stays masked; out_conf = c_i (0 at positions that were not masked);
- * exempt (nullable) = 1 where the decision lies within 1e-5 of the threshold
- * or of the k-th / (k+1)-th confidence.                                     */
+ * exempt (nullable) = 1 where the decision lies within 1e-5 of the threshold,
+ * or where the count rule decides and the confidence just across the top-k
+ * boundary is within 1e-5.                                                   */
 typedef struct { double c; int pos; } conf_pos;
 
 static int more_confident_first(const void *x, const void *y)
@@ -482,9 +485,10 @@ void dd_oracle_unmask(const uint16_t *logits, const int32_t *tokens, const uint8
             if (unmask) out_tokens[t] = best[t];
             if (exempt) {
                 int near = fabs(order[r].c - tau) <= EXEMPT_BAND;
-                if (!above && k > 0 && k < n) {      /* the top-k boundary decides */
-                    if (fabs(order[r].c - order[k - 1].c) <= EXEMPT_BAND) near = 1;
-                    if (fabs(order[r].c - order[k].c) <= EXEMPT_BAND) near = 1;
+                if (!above && k > 0 && k < n) {      /* the top-k boundary decides: uncertain only if
+                                                        the confidence across the boundary is within the band */
+                    if (r < k && fabs(order[r].c - order[k].c) <= EXEMPT_BAND) near = 1;
+                    if (r >= k && fabs(order[r].c - order[k - 1].c) <= EXEMPT_BAND) near = 1;
                 }
                 exempt[t] = (uint8_t)near;
             }
