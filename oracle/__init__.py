@@ -204,3 +204,47 @@ def unmask(logits, tokens, flags, tau, k):
     _load().dd_oracle_unmask(_ptr(logits), _ptr(tokens), _ptr(flags), tau32, int(k),
                              _ptr(out_tokens), _ptr(out_mask), _ptr(out_conf), _ptr(exempt), B, P, V)
     return dict(out_tokens=out_tokens, out_mask=out_mask, out_conf=out_conf, exempt=exempt)
+
+
+def dualdiffusion_loop(drafter, verifier, tokens, mask_id, K, mode, tau, k, seed=0,
+                       unmask_tau=float("inf"), unmask_k=1, max_cycles=10_000):
+    """Algorithm 1 with the oracle's own Unmask and verification steps (numpy arrays throughout).
+
+    drafter, verifier: callables tokens int32 [B,P] -> logits uint16 [B,P,V] (bf16 bits).
+    Returns (tokens, dict of counters, number of decisions the oracle flagged as lying within
+    its exemption band)."""
+    x = np.array(tokens, dtype=np.int32, copy=True)
+    stats = dict(cycles=0, drafter_calls=0, verifier_calls=0, unmasked_by_drafter=0,
+                 remasked_by_verifier=0, masked_after_cycle=[])
+    near = 0
+    while stats["cycles"] < max_cycles:
+        masked = x == mask_id
+        if not masked.any():
+            break
+        drafted = np.zeros_like(masked)
+        for _ in range(K):                                   # drafting phase
+            if not masked.any():
+                break
+            r = unmask(drafter(x), x, masked.astype(np.uint8), unmask_tau, unmask_k)
+            stats["drafter_calls"] += 1
+            still = r["out_mask"].astype(bool)
+            newly = masked & ~still
+            drafted |= newly
+            stats["unmasked_by_drafter"] += int(newly.sum())
+            near += int(r["exempt"].sum())
+            x = r["out_tokens"]
+            masked = still
+        logits_v = verifier(x)                               # verification phase
+        stats["verifier_calls"] += 1
+        logits_d = None
+        if (mode & 0xFF) == 1:
+            logits_d = drafter(x)
+            stats["drafter_calls"] += 1
+        r = verify(logits_d, logits_v, x, drafted.astype(np.uint8), mode, tau, k, seed + stats["cycles"])
+        near += int(r["exempt"].sum())
+        remask = r["out_mask"].astype(bool)
+        x = np.where(remask, np.int32(mask_id), r["out_tokens"]).astype(np.int32)
+        stats["remasked_by_verifier"] += int(remask.sum())
+        stats["cycles"] += 1
+        stats["masked_after_cycle"].append(int((x == mask_id).sum()))
+    return x, stats, near
