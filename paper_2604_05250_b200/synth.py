@@ -164,14 +164,16 @@ class ToyModel:
     """
 
     def __init__(self, target, V, mask_id, seed, wrong_share=0.0, base=2.0, gain=6.0):
+        assert mask_id == V - 1 and int(np.max(target)) < V - 1, "tokens 0..V-2, the mask id is V-1"
         rng = np.random.default_rng([int(seed), 0x70F])
         B, P = target.shape
         self.mask_id = int(mask_id)
         self.noise = rng.standard_normal((B, P, V), dtype=np.float32)
         self.belief = np.array(target, dtype=np.int64, copy=True)
         wrong = rng.random((B, P)) < wrong_share
-        shift = rng.integers(1, V, size=(B, P))
-        self.belief[wrong] = (self.belief[wrong] + shift[wrong]) % V
+        # a wrong belief is another ordinary token (the mask id, the last of the vocabulary, is none)
+        shift = rng.integers(1, V - 1, size=(B, P))
+        self.belief[wrong] = (self.belief[wrong] + shift[wrong]) % (V - 1)
         self.jitter = rng.random((B, P)).astype(np.float32)
         self.base, self.gain = np.float32(base), np.float32(gain)
 
