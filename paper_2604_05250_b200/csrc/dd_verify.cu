@@ -203,12 +203,14 @@ bool streaming_path(const void *drafter, const void *verifier, int V, bool kl)
 // Streaming path: pieces per chunk.  Every streaming warp of a CTA takes whole (row, chunk)
 // units in turn, so a CTA's time is rounds * pieces-per-unit; pick the unit size that wastes
 // least for `rows` flagged rows on `ctas` CTAs (a smaller unit only if it saves 5 %), among
-// those whose partials fit `max_partials` (0: no limit).
-int pick_pieces(int V, long rows, int ctas, long max_partials)
+// those whose partials fit `max_partials` (0: no limit).  `even`: only even counts (without a
+// drafter tensor a warp steps through its unit two pieces at a time).
+int pick_pieces(int V, long rows, int ctas, long max_partials, bool even)
 {
     int best = kMaxPiecesPerChunk;
     long best_cost = -1;
     for (int k = kMaxPiecesPerChunk; k >= kMinPiecesPerChunk; --k) {
+        if (even && (k & 1)) continue;
         const long nch = (V + (long)k * kPiece - 1) / ((long)k * kPiece);
         if (max_partials > 0 && rows * nch > max_partials && k != kMaxPiecesPerChunk) continue;
         const long per_cta = (rows * nch + ctas - 1) / ctas;
@@ -339,7 +341,7 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     if (streaming) {
         const int sms = sm_count_of_current_device();
         if (sms < 0) return sms;
-        pieces = pick_pieces(V, (long)B * P, sms, (1L << 31) - 1);
+        pieces = pick_pieces(V, (long)B * P, sms, (1L << 31) - 1, !kl);
     }
     chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
     if ((long)B * P * p.nchunks >= (1L << 31)) return DD_ERR_UNSUPPORTED;
@@ -444,7 +446,7 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     if (streaming) {
         const int sms = sm_count_of_current_device();
         if (sms < 0) return sms;
-        pieces = pick_pieces(V, (long)B * P, sms, kStaticMaxPartials);
+        pieces = pick_pieces(V, (long)B * P, sms, kStaticMaxPartials, !kl);
     }
     chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
     if ((long)B * P * p.nchunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;

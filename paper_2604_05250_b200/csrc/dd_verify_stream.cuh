@@ -5,7 +5,8 @@
 // range come out in whole rounds of the streaming warps) are numbered in row order and cut into equal
 // contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  The
 // range's units go to the streaming warps in turn.  A warp walks its unit in pieces of 1024
-// logits per tensor: every lane holds four 16-byte vectors per tensor of the current piece
+// logits per tensor (2048 of the verifier when there is no drafter tensor): every lane holds
+// four 16-byte vectors per tensor of the current piece (eight of the verifier)
 // in registers and has the loads of the next piece in flight while it computes (the
 // measured copy bandwidth is reached with this depth; a shared-memory ring fed by bulk
 // copies reached it too but cost about four times the instructions per piece).  Within a
@@ -34,6 +35,14 @@ constexpr int kSChunk = kPiece * kMaxPiecesPerChunk;
 constexpr int kSTable = 768;                                  // chunk partials a CTA keeps per range
 constexpr unsigned kErrWaitQueue = 0x800;
 
+// Logits per tensor in one step of a warp.  Without a drafter tensor (TRUST, CONF) the registers
+// that would hold the drafter's vectors hold four more vectors of the verifier: the piece is twice
+// as long, so that a warp has as many bytes in flight as in KL mode.
+template <bool KL>
+struct PieceOf {
+    static constexpr int value = KL ? kPiece : 2 * kPiece;
+};
+
 __device__ __forceinline__ uint4 ld_stream(const uint4 *ptr)
 {
     uint4 r;
@@ -59,7 +68,8 @@ __device__ __forceinline__ void lane_reset(LaneState &L)
 }
 
 // One piece (n logits, a multiple of 8; lane's vector j covers logits (lane + 32 j) * 8 ..+7).
-// kFull: n == kPiece, no vector is absent.
+// KL: rv / rd are the verifier's / drafter's vectors 0..3.  Otherwise rv holds the verifier's
+// vectors 0..3 and rd its vectors 4..7.  kFull: no vector is absent.
 template <bool KL, bool kFull>
 __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecPerThread],
                                            const uint4 (&rd)[kVecPerThread], int n, int lane, int ordinal)
@@ -86,12 +96,30 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
             }
         }
     }
+    if (!KL) {
+        // the verifier's vectors 4..7, after 0..3: words are visited in the order of their logits,
+        // so a maximum that occurs twice keeps its first place
+#pragma unroll
+        for (int j = 0; j < kVecPerThread; ++j) {
+            const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const __nv_bfloat162 w = *reinterpret_cast<const __nv_bfloat162 *>(&wd[h]);
+                const __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162 *>(&max2_v);
+                const uint32_t rose = __hgt2_mask(w, m);
+                const __nv_bfloat162 m_new = __hmax2(m, w);
+                max2_v = *reinterpret_cast<const uint32_t *>(&m_new);
+                const uint32_t q2 = (uint32_t)((kVecPerThread + j) * 4 + h) * 0x00010001u;
+                where2 = (where2 & ~rose) | (q2 & rose);
+            }
+        }
+    }
     {
         // halves that rose during this piece take (piece ordinal, word ordinal)
         const __nv_bfloat162 before = *reinterpret_cast<const __nv_bfloat162 *>(&L.max2_v);
         const __nv_bfloat162 after = *reinterpret_cast<const __nv_bfloat162 *>(&max2_v);
         const uint32_t rose = __hgt2_mask(after, before);
-        const uint32_t q2 = where2 + (uint32_t)(ordinal * 16) * 0x00010001u;
+        const uint32_t q2 = where2 + (uint32_t)(ordinal * (KL ? 16 : 32)) * 0x00010001u;
         L.where2_v = (L.where2_v & ~rose) | (q2 & rose);
         L.max2_v = max2_v;
         L.max2_d = max2_d;
@@ -136,6 +164,20 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
             }
         }
     }
+    if (!KL) {
+#pragma unroll
+        for (int j = 0; j < kVecPerThread; ++j) {
+            if (kFull || (lane + (kVecPerThread + j) * 32) * 8 < n) {
+                const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float2 v2 = make_float2(bf16lo(wd[h]), bf16hi(wd[h]));
+                    const float2 a = __ffma2_rn(v2, log2e2, nMv2);
+                    s_v = __fadd2_rn(s_v, make_float2(ex2_approx(a.x), ex2_approx(a.y)));
+                }
+            }
+        }
+    }
     L.s_v = s_v; L.s_d = s_d; L.t = t;
 }
 
@@ -146,9 +188,10 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
 {
     Partial c;
     const float lo_m = bf16lo(L.max2_v), hi_m = bf16hi(L.max2_v);
-    auto element_of = [&](uint32_t q, int odd) {     // q = piece * 16 + j * 4 + h
-        return chunk_begin + (int)(q >> 4) * kPiece + (lane + 32 * (int)((q >> 2) & 3u)) * 8 +
-               2 * (int)(q & 3u) + odd;
+    auto element_of = [&](uint32_t q, int odd) {     // q = piece * 16 + j * 4 + h (KL), piece * 32 + j * 4 + h
+        const int piece = KL ? (int)(q >> 4) : (int)(q >> 5);
+        const int vec = KL ? (int)((q >> 2) & 3u) : (int)((q >> 2) & 7u);
+        return chunk_begin + piece * PieceOf<KL>::value + (lane + 32 * vec) * 8 + 2 * (int)(q & 3u) + odd;
     };
     const int e_lo = element_of(L.where2_v & 0xFFFFu, 0), e_hi = element_of(L.where2_v >> 16, 1);
     const float my_m = fmaxf(lo_m, hi_m);

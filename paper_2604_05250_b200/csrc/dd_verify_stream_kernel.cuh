@@ -224,8 +224,9 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
 
         // =================================================================== streaming warps
         const unsigned ulo = (unsigned)lo, uhi = (unsigned)hi, uflo = (unsigned)f_lo;   // units fit 31 bits
-        const int chunk_len = p.chunk, chunk_pieces = p.chunk / kPiece;                 // logits, pieces per chunk
-        const int last_pieces = (p.V - (nch - 1) * chunk_len + kPiece - 1) / kPiece;       // of a row's last chunk
+        constexpr int kStep = PieceOf<KL>::value;                                        // logits per piece
+        const int chunk_len = p.chunk, chunk_pieces = p.chunk / kStep;                  // logits, pieces per chunk
+        const int last_pieces = (p.V - (nch - 1) * chunk_len + kStep - 1) / kStep;         // of a row's last chunk
 
         // Units of the range go to the streaming warps in turn: warp w takes units w, w + 15, ...
         // A cursor walks one warp's pieces in order (all lanes hold the same values).
@@ -251,34 +252,28 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             }
             enter_unit(c);
         };
-        // the lane's vectors of the cursor's piece: four per tensor, -inf where the row has ended
+        // the lane's vectors of the cursor's piece, -inf where the row has ended: four per tensor, or
+        // (no drafter tensor) eight of the verifier, the second four in d
         auto fetch = [&](const Cursor &c, uint4 (&v)[kVecPerThread], uint4 (&d)[kVecPerThread]) {
-            const int e_begin = c.chunk * chunk_len + c.piece * kPiece;
+            const int e_begin = c.chunk * chunk_len + c.piece * kStep;
             const int n = p.V - e_begin;                      // logits left in the row
             const size_t off = (size_t)c.row * p.V + e_begin;
             const uint4 *gv = reinterpret_cast<const uint4 *>(p.verifier + off) + lane;
-            const uint4 *gd = reinterpret_cast<const uint4 *>(p.drafter + off) + lane;
-            if (n >= kPiece) {
+            const uint4 *gd = KL ? reinterpret_cast<const uint4 *>(p.drafter + off) + lane : gv + 32 * kVecPerThread;
+            if (n >= kStep) {
 #pragma unroll
                 for (int j = 0; j < kVecPerThread; ++j) {
                     v[j] = ld_stream(gv + 32 * j);
-                    if (KL) d[j] = ld_stream(gd + 32 * j);
+                    d[j] = ld_stream(gd + 32 * j);
                 }
             } else {
 #pragma unroll
                 for (int j = 0; j < kVecPerThread; ++j) {
-                    const bool in = (lane + 32 * j) * 8 < n;
                     v[j] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-                    if (KL) d[j] = v[j];
-                    if (in) {
-                        v[j] = ld_stream(gv + 32 * j);
-                        if (KL) d[j] = ld_stream(gd + 32 * j);
-                    }
+                    d[j] = v[j];
+                    if ((lane + 32 * j) * 8 < n) v[j] = ld_stream(gv + 32 * j);
+                    if ((lane + 32 * (KL ? j : kVecPerThread + j)) * 8 < n) d[j] = ld_stream(gd + 32 * j);
                 }
-            }
-            if (!KL) {
-#pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) d[j] = make_uint4(0u, 0u, 0u, 0u);
             }
         };
 
@@ -304,8 +299,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             advance(nc);
             if (nc.t < n_units) fetch(nc, nv, nd);            // in flight while this piece is computed
 
-            const int n = min(kPiece, p.V - (cc.chunk * chunk_len + cc.piece * kPiece));
-            if (n == kPiece) lane_piece<KL, true>(L, rv, rd, n, lane, cc.piece);
+            const int n = min(kStep, p.V - (cc.chunk * chunk_len + cc.piece * kStep));
+            if (n == kStep) lane_piece<KL, true>(L, rv, rd, n, lane, cc.piece);
             else lane_piece<KL, false>(L, rv, rd, n, lane, cc.piece);
             const bool chunk_ends = cc.piece == cc.npieces - 1;
             const Cursor done = cc;
