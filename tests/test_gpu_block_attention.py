@@ -122,3 +122,15 @@ def test_argument_errors(dd):
     assert L.dd_block_attention(p(q), p(k), p(k), p(q), 1, 2, 0, 32, 128, None, 0, 0.1, None) == dd.DD_ERR_INVALID_ARG
     assert L.dd_block_attention(p(q), p(k), p(k), p(q), 1, 2, 16, 32, 96, None, 0, 0.1, None) == dd.DD_ERR_UNSUPPORTED
     assert L.dd_block_attention(None, p(k), p(k), p(q), 1, 2, 16, 32, 128, None, 0, 0.1, None) == dd.DD_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("layout", ["bhnd", "bnhd"])
+def test_drafter_shape_full_size(dd, oracle_mod, layout):
+    """The shape bench_ops times: 32 queries over 1024 stored keys, B = 16, H = 32, D = 128."""
+    B, H, Nq, Nkv, D = 16, 32, 32, 1024, 128
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 77)
+    kv_len = np.random.default_rng(3).integers(Nkv // 4, Nkv + 1, size=B).astype(np.int32)
+    if layout == "bnhd":
+        q, k, v = (np.ascontiguousarray(a.transpose(0, 2, 1, 3)) for a in (q, k, v))
+    got = run_gpu(dd, q, k, v, D ** -0.5, kv_len=kv_len, layout=layout)
+    check_attention(got, oracle_mod.block_attention(q, k, v, D ** -0.5, kv_len=kv_len, layout=layout))

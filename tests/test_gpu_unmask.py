@@ -65,3 +65,10 @@ def test_nothing_masked_passes_through(dd, oracle_mod):
     flags[1] = 0
     ref, om = compare(dd, oracle_mod, logits, flags, 0.4, 2)
     assert not om[1].any()
+
+
+def test_batched_serving_shape(dd, oracle_mod):
+    """The cfg2 logits shape [16,256,126464] with 25-100 % of the positions masked per sequence."""
+    _, logits, _, flags = synth.verify_config_inputs(2)
+    ref, om = compare(dd, oracle_mod, logits, flags, 0.5, 16)
+    assert ((flags == 1) & (om == 0)).sum(axis=1).min() >= 16
