@@ -32,8 +32,6 @@ def problem(seed, B=3, P=40, prompt=8):
 
 
 def on_device(model):
-    import torch
-
     def call(tokens):
         return to_torch_bf16(model(tokens.cpu().numpy()), "cuda")
     return call
