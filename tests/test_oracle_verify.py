@@ -309,6 +309,21 @@ def test_exemption_flags_mark_topk_boundary(oracle_mod):
     assert list(r["exempt"][0]) == [1, 1, 0, 0]       # the tied pair straddles the boundary
 
 
+def test_well_separated_topk_boundary_is_not_exempt(oracle_mod):
+    """Confidences 0.88, 0.73, 0.95, 0.62 (two-token rows with peaks 2, 1, 3, 0.5): every position
+    fails tau = 0.999 and k = 2 keeps positions 2 and 0.  No reliability is within 1e-5 of the one
+    across the boundary, so nothing is exempt, the positions at the boundary included."""
+    ver = bits(np.array([[[0.0, 2.0], [0.0, 1.0], [0.0, 3.0], [0.0, 0.5]]]))
+    tokens = np.zeros((1, 4), dtype=np.int32)
+    flags = np.ones((1, 4), dtype=np.uint8)
+    r = oracle_mod.verify(None, ver, tokens, flags, CONF, 0.999, 2, 0)
+    assert list(r["out_mask"][0]) == [0, 1, 0, 1]
+    assert list(r["exempt"][0]) == [0, 0, 0, 0]
+    u = oracle_mod.unmask(ver, tokens, flags, np.inf, 2)
+    assert list(u["out_mask"][0]) == [0, 1, 0, 1]
+    assert list(u["exempt"][0]) == [0, 0, 0, 0]
+
+
 def test_unknown_mode_rejected(oracle_mod):
     dra, ver, tokens, flags = tiny_case(P=2, V=4)
     with pytest.raises(ValueError):
