@@ -444,16 +444,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 for (int j = 0; j < nkv && err == 0; ++j) {
                     const int item_v = 2 * j + 1, item_k = 2 * j + 2;
                     const bool more = j + 1 < nkv;
+                    // both tiles this round reads are waited for here, not between two groups of MMAs:
+                    // a wait in between lets the tensor core run dry
                     if (!wait_item(item_v)) { err = kErrWaitKV; break; }
+                    if (more && !wait_item(item_k)) { err = kErrWaitKV; break; }
                     for (int g = 0; g < ntiles; ++g) {
                         if (!mbar_wait(bar_p_full(g), j & 1)) { err = kErrWaitP; break; }
                         tc_fence_after();
                         issue_o(g, item_v % kStages, j == 0);
-                        if (more) {
-                            if (g == 0 && !wait_item(item_k)) { err = kErrWaitKV; break; }
-                            tc_fence_after();
-                            issue_s(g, item_k % kStages);
-                        }
+                        if (more) issue_s(g, item_k % kStages);
                     }
                     if (err) break;
                     mma_commit(bar_kv_empty(item_v % kStages));
