@@ -268,6 +268,9 @@ void dd_oracle_row_scores(const uint16_t *drafter_row, const uint16_t *verifier_
         for (int x = 0; x < V; ++x) {
             const double log_pd = bf16_to_f64(drafter_row[x]) - lse_d;
             const double log_pv = bf16_to_f64(verifier_row[x]) - lse_v;
+            /* a token the drafter excludes (logit -inf, p_D(x) = 0) adds nothing: the
+             * Kullback-Leibler sum of Eq. 5 runs over the support of p_D (0 ln 0 = 0) */
+            if (log_pd == -INFINITY) continue;
             acc += exp(log_pd) * (log_pd - log_pv);
         }
         if (acc < 0.0) acc = 0.0;

@@ -256,6 +256,25 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                  : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
                 }
                 l_run += sum;
+                if (kBlock && masked) {
+                    // Keys past the end of the sequence have weight zero, but 0 x NaN is NaN in the
+                    // product P V, and padding may hold any bit pattern: clear their value rows in
+                    // the ring slot (whole 128-byte rows, which the swizzle maps onto themselves)
+                    // before the weights are handed over.  The slot cannot be refilled before this
+                    // group's product has read it.
+                    const int item_v = 2 * j + 1, slot_v = item_v % kStages;
+                    if (!mbar_wait(bar_kv_full(slot_v), (item_v / kStages) & 1)) { err = kErrWaitKV; break; }
+                    const int r = (warp & 3) * 32 + lane;
+                    if (r >= valid) {
+                        const uint32_t row = sRing + slot_v * kTileBytes + r * 128;
+#pragma unroll
+                        for (int cx = 0; cx < kBoxes; ++cx)
+#pragma unroll
+                            for (int c16 = 0; c16 < 8; ++c16)
+                                st_shared_v4(row + cx * kBoxBytes + c16 * 16, 0u, 0u, 0u, 0u);
+                    }
+                    fence_proxy_async_smem();
+                }
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar_p_full(g));

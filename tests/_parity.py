@@ -59,3 +59,41 @@ def check_verify(gpu_tokens, gpu_mask, gpu_score, ref, flags, tokens_in):
     assert (gpu_tokens[~flags] == tokens_in[~flags]).all()
     assert not gpu_mask[~flags].any() and not gpu_score[~flags].any()
     return int(exempt.sum())
+
+
+# ----------------------------------------------------------------------------- guard regions
+#
+# Every GPU output is allocated inside a larger buffer filled with a sentinel; after the call the
+# margins must be untouched.  An out-of-range store by a kernel (a decision stage that runs past
+# the sequence, an epilogue tile that is not clipped) then fails the test that made it.
+
+GUARD_ELEMS = 1024          # per side; a multiple of 8, so 2-byte views stay 16-byte aligned
+
+
+class Guarded:
+    """A device (or pinned host) tensor of `shape` with GUARD_ELEMS sentinel elements on both sides."""
+
+    _SENTINEL = {"torch.bfloat16": -2.0078125e3, "torch.float32": -7.25e11, "torch.int32": -0x5A5A5A5B,
+                 "torch.uint8": 0xA5}
+
+    def __init__(self, shape, dtype, device="cuda", pin=False):
+        import torch
+        n = int(np.prod(shape))
+        self.fill = self._SENTINEL[str(dtype)]
+        if device is None:
+            self.raw = torch.empty(n + 2 * GUARD_ELEMS, dtype=dtype)
+            if pin:
+                self.raw = self.raw.pin_memory()
+        else:
+            self.raw = torch.empty(n + 2 * GUARD_ELEMS, dtype=dtype, device=device)
+        self.raw.fill_(self.fill)
+        self.view = self.raw[GUARD_ELEMS:GUARD_ELEMS + n].view(*shape)
+        self.n = n
+
+    def check(self, what="output"):
+        import torch
+        lo = self.raw[:GUARD_ELEMS]
+        hi = self.raw[GUARD_ELEMS + self.n:]
+        ref = torch.full_like(lo, self.fill)
+        assert torch.equal(lo, ref), f"{what}: the kernel wrote below the buffer"
+        assert torch.equal(hi, ref), f"{what}: the kernel wrote past the buffer"

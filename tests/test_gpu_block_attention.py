@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from paper_2604_05250_b200 import synth
-from tests._parity import bf16_tensor_to_f64, check_attention, to_torch_bf16
+from tests._parity import Guarded, bf16_tensor_to_f64, check_attention, to_torch_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -34,9 +34,11 @@ def run_gpu(dd, q, k, v, scale, kv_len=None, layout="bhnd"):
     import torch
     tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
     tl = None if kv_len is None else torch.from_numpy(np.asarray(kv_len, dtype=np.int32)).cuda()
-    out = dd.block_attention(tq, tk, tv, kv_len=tl, layout=layout, scale=scale)
+    g = Guarded(tq.shape, torch.bfloat16)        # guard regions on both sides of the output
+    out = dd.block_attention(tq, tk, tv, out=g.view, kv_len=tl, layout=layout, scale=scale)
     torch.cuda.synchronize()
     assert dd.attention_status() == 0
+    g.check("block attention output")
     return bf16_tensor_to_f64(out)
 
 
@@ -68,6 +70,27 @@ def test_ragged_key_counts_and_padding(dd, oracle_mod):
     # lengths outside [0, Nkv] are clamped
     got2 = run_gpu(dd, q, k, v, D ** -0.5, kv_len=np.array([9999, 1, 128, 129, -5, 511], dtype=np.int32))
     np.testing.assert_array_equal(got2, got)
+
+
+@pytest.mark.parametrize("layout", ["bhnd", "bnhd"])
+def test_padding_of_nan_and_inf_never_contributes(dd, oracle_mod, layout):
+    """Keys and values beyond n_b are padding (Eq. 3 runs over the keys that exist): a cache
+    that was never initialised there may hold any bit pattern, NaN and infinities included."""
+    B, H, Nq, Nkv, D = 5, 2, 150, 520, 128
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 23)
+    kv_len = np.array([520, 1, 129, 383, 512], dtype=np.int32)
+    junk = np.array([0x7FC0, 0x7F80, 0xFF80, 0xFFFF], dtype=np.uint16)       # NaN, +inf, -inf, NaN
+    for b in range(B):
+        n = Nkv - kv_len[b]
+        k[b, :, kv_len[b]:] = junk[np.arange(n * D).reshape(n, D) % 4]
+        v[b, :, kv_len[b]:] = junk[(np.arange(n * D).reshape(n, D) + 1) % 4]
+    ref = oracle_mod.block_attention(q, k, v, D ** -0.5, kv_len=kv_len)
+    assert np.isfinite(ref).all()
+    if layout == "bnhd":
+        q, k, v = (np.ascontiguousarray(a.transpose(0, 2, 1, 3)) for a in (q, k, v))
+        ref = np.ascontiguousarray(ref.transpose(0, 2, 1, 3))
+    got = run_gpu(dd, q, k, v, D ** -0.5, kv_len=kv_len, layout=layout)
+    check_attention(got, ref)
 
 
 @pytest.mark.parametrize("D", [64, 128])

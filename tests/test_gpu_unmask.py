@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 from paper_2604_05250_b200 import synth
-from tests._parity import SCORE_ABS_FLOOR, SCORE_REL, to_torch_bf16
+from tests._parity import SCORE_ABS_FLOOR, SCORE_REL, Guarded, to_torch_bf16
 
 pytestmark = pytest.mark.gpu
 MASK_ID = 126336
@@ -25,10 +25,14 @@ def compare(dd, oracle_mod, logits, flags, tau, k):
     tokens = np.full((B, P), MASK_ID, dtype=np.int32)
     tokens[flags == 0] = 5
     ref = oracle_mod.unmask(logits, tokens, flags, tau, k)
+    g_tok, g_mask = Guarded((B, P), torch.int32), Guarded((B, P), torch.uint8)
+    g_conf = Guarded((B, P), torch.float32)
     ot, om, oc = dd.unmask(to_torch_bf16(logits, "cuda"), torch.from_numpy(tokens).cuda(),
-                           torch.from_numpy(flags).cuda(), tau, k)
+                           torch.from_numpy(flags).cuda(), tau, k, out_tokens=g_tok.view, out_mask=g_mask.view,
+                           out_conf=g_conf.view)
     torch.cuda.synchronize()
     assert dd.verify_status() == 0
+    g_tok.check("out_tokens"); g_mask.check("out_mask"); g_conf.check("out_conf")
     ot, om, oc = ot.cpu().numpy(), om.cpu().numpy(), oc.cpu().numpy().astype(np.float64)
     tol = np.maximum(SCORE_REL * np.abs(ref["out_conf"]), SCORE_ABS_FLOOR)
     assert (np.abs(oc - ref["out_conf"]) <= tol).all()

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 from paper_2604_05250_b200 import synth
-from tests._parity import check_verify, to_torch_bf16
+from tests._parity import Guarded, check_verify, to_torch_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -32,8 +32,15 @@ def run_gpu(dd, dra, ver, tokens, flags, mode, tau, k, seed, host=False):
         t_tok, t_fl = t_tok.pin_memory(), t_fl.pin_memory()
     else:
         t_tok, t_fl = t_tok.cuda(), t_fl.cuda()
-    ot, om, osc = dd.verify(t_dra, t_ver, t_tok, t_fl, mode, tau, k, seed, host=host)
+    # each output sits between two guard regions that the kernels must leave alone
+    g_tok = Guarded(tokens.shape, torch.int32, device=dev, pin=host)
+    g_mask = Guarded(tokens.shape, torch.uint8, device=dev, pin=host)
+    g_score = Guarded(tokens.shape, torch.float32, device=dev, pin=host)
+    ot, om, osc = dd.verify(t_dra, t_ver, t_tok, t_fl, mode, tau, k, seed, out_tokens=g_tok.view,
+                            out_mask=g_mask.view, out_score=g_score.view, host=host)
     torch.cuda.synchronize()
+    assert dd.verify_status() == 0
+    g_tok.check("out_tokens"); g_mask.check("out_mask"); g_score.check("out_score")
     return ot.cpu().numpy(), om.cpu().numpy(), osc.cpu().numpy()
 
 

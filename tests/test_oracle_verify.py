@@ -143,6 +143,31 @@ def test_matches_library_log_softmax_and_rel_entr(oracle_mod, V):
         assert a == int(np.argmax(f64(v[i])))
 
 
+def test_tokens_the_drafter_excludes_add_nothing(oracle_mod):
+    """Logit -inf (a banned or padded vocabulary entry) is p(x) = 0.  Eq. 5 is a sum over the
+    support of p_D (0 ln 0 = 0): an entry the drafter excludes contributes no term, an entry both
+    models exclude might as well not exist, an entry only the verifier excludes makes the
+    divergence infinite."""
+    V = 40
+    d = f64(rand_rows(1, V, 8)[0])
+    v = f64(rand_rows(1, V, 9)[0])
+    d[[3, 17, 30]] = -np.inf
+    v[[17, 30]] = -np.inf               # excluded by both
+    a, c, kl = oracle_mod.row_scores(bits(d), bits(v))
+    lp_d = scipy.special.log_softmax(f64(bits(d)))
+    lp_v = scipy.special.log_softmax(f64(bits(v)))
+    ref = scipy.special.rel_entr(np.exp(lp_d), np.exp(lp_v)).sum()
+    assert np.isfinite(kl) and abs(kl - ref) < 1e-12
+    # without the entries both models exclude, the same rows give the same number
+    keep = np.isfinite(d) | np.isfinite(v)
+    assert keep.sum() == V - 2
+    sub = oracle_mod.row_scores(bits(d[keep]), bits(v[keep]))[2]
+    assert abs(kl - sub) < 1e-12
+    assert abs(c - np.exp(lp_v).max()) < 1e-14 and a == int(np.argmax(f64(bits(v))))
+    v[5] = -np.inf                      # p_D(5) > 0 = p_V(5)
+    assert oracle_mod.row_scores(bits(d), bits(v))[2] == np.inf
+
+
 def test_argmax_lowest_index_on_ties(oracle_mod):
     row = np.zeros(100, dtype=np.float32)
     row[[13, 57, 99]] = 9.0
@@ -322,6 +347,40 @@ def test_well_separated_topk_boundary_is_not_exempt(oracle_mod):
     u = oracle_mod.unmask(ver, tokens, flags, np.inf, 2)
     assert list(u["out_mask"][0]) == [0, 1, 0, 1]
     assert list(u["exempt"][0]) == [0, 0, 0, 0]
+
+
+# Seeds whose uniform for (b, i) = (0, 0) lies next to 1/2: found by a search over the Philox
+# mapping pinned above; the tests re-check the distance before using them.
+SEEDS_NEAR_HALF = {41794: -4.47e-6, 95032: 3.76e-6}       # inside the 1e-5 band
+SEEDS_OFF_HALF = {1782: -4.31e-5, 3545: 2.84e-5}          # outside it
+
+
+@pytest.mark.parametrize("seed,delta,inside", [(s, d, True) for s, d in SEEDS_NEAR_HALF.items()] +
+                         [(s, d, False) for s, d in SEEDS_OFF_HALF.items()])
+def test_probabilistic_rules_exemption_band(oracle_mod, seed, delta, inside):
+    """The probabilistic rules flag a decision as exempt iff the uniform lies within 1e-5 of the
+    remask probability (1 - c for confidence, Eq. 6's share for KL); both are 1/2 exactly here."""
+    u0 = oracle_mod.uniform(seed, 0, 0)
+    assert abs((u0 - 0.5) - delta) < 1e-7 and (abs(u0 - 0.5) <= 1e-5) == inside
+    # confidence: two tokens with equal logits, c = 1/2, remask iff u < 1/2
+    ver = bits(np.zeros((1, 1, 2)))
+    tokens = np.array([[1]], dtype=np.int32)
+    flags = np.ones((1, 1), dtype=np.uint8)
+    r = oracle_mod.verify(None, ver, tokens, flags, CONF | PROB, 0.9, 0, seed)
+    assert r["out_score"][0, 0] == 0.5
+    assert r["out_mask"][0, 0] == (1 if u0 < 0.5 else 0)
+    assert r["exempt"][0, 0] == (1 if inside else 0)
+    # KL: two positions with the same pair of rows share Eq. 6's mass equally
+    dra = bits(np.array([[[2.0, 0.0], [2.0, 0.0]]]))
+    ver = bits(np.zeros((1, 2, 2)))
+    tokens = np.array([[0, 0]], dtype=np.int32)
+    flags = np.ones((1, 2), dtype=np.uint8)
+    r = oracle_mod.verify(dra, ver, tokens, flags, KL | PROB, 0.0, 0, seed)
+    assert r["out_score"][0, 0] == r["out_score"][0, 1] > 0
+    u1 = oracle_mod.uniform(seed, 0, 1)
+    assert abs(u1 - 0.5) > 1e-3                         # the second position is far from the boundary
+    assert r["out_mask"][0].tolist() == [int(u0 < 0.5), int(u1 < 0.5)]
+    assert r["exempt"][0].tolist() == [1 if inside else 0, 0]
 
 
 def test_unknown_mode_rejected(oracle_mod):
