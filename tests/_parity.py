@@ -1,6 +1,9 @@
 """Shared comparison rules of the GPU parity tests.
 
-Attention: max-abs <= 1e-2 and mean-abs <= 1e-3 against the fp64 oracle.
+Attention: max-abs <= 1e-2 and mean-abs <= 1e-3 against the fp64 oracle.  The output is
+bf16: from |out| = 4 upwards its grid is coarser than 2 x 1e-2 (spacing 2^-5 in [4, 8)), so
+that no bf16 value need lie within 1e-2 of the exact result; there the max-abs bar scales with
+the spacing (2e-2 in [4, 8), 4e-2 in [8, 16), ...).  Below 4 it is 1e-2 as stated.
 Verify: scores within 1e-4 relative (absolute floor 1e-6 where the score is
 near zero); remask sets and emitted tokens bit-exact except at positions the
 oracle flags as lying within 1e-5 of a decision boundary.
@@ -26,10 +29,18 @@ def bf16_tensor_to_f64(t):
     return t.detach().to("cpu").to(torch.float64).numpy()
 
 
+def attention_max_abs_bar(oracle_out):
+    """1e-2, times the bf16 grid spacing relative to that of [2, 4) where the exact value is >= 4."""
+    mag = np.maximum(np.abs(oracle_out), 1e-30)
+    return ATTN_MAX_ABS * np.maximum(1.0, np.exp2(np.floor(np.log2(mag)) - 1.0))
+
+
 def check_attention(gpu_out_f64, oracle_out):
     diff = np.abs(gpu_out_f64 - oracle_out)
     assert np.isfinite(gpu_out_f64).all()
-    assert diff.max() <= ATTN_MAX_ABS, f"max-abs {diff.max():.3e}"
+    over = diff > attention_max_abs_bar(oracle_out)
+    assert not over.any(), (f"{over.sum()} elements over the max-abs bar; worst {diff[over].max():.3e} "
+                            f"at |exact| = {np.abs(oracle_out)[over][diff[over].argmax()]:.3f}")
     assert diff.mean() <= ATTN_MEAN_ABS, f"mean-abs {diff.mean():.3e}"
     return float(diff.max()), float(diff.mean())
 
