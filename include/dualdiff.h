@@ -178,8 +178,9 @@ int dd_verify_host(const void *drafter_logits, const void *verifier_logits,
  * fixed memory budget, that may not trigger the device-wide synchronisation of
  * cudaMalloc/cudaFree, or that does not own the allocator of its process: this
  * call performs no cudaMalloc, cudaFree or other allocating routine.  Its scratch
- * (chunk partials, row results, completion counters) is a fixed array of about
- * 2.1 MB inside the library, held by every GPU that loads the library until the
+ * (chunk partials, row results, completion counters, and a health word of its
+ * own that dd_verify_status reads as well) is a fixed array of about 2.1 MB
+ * inside the library, held by every GPU that loads the library until the
  * process exits.
  * Limits: B*P <= 4096 and B*P*ceil(V/8192) <= 65536; larger problems return
  * DD_ERR_UNSUPPORTED and launch nothing.
@@ -194,6 +195,16 @@ int dd_verify_static(const void *drafter_logits, const void *verifier_logits,
                      int mode, float tau, int k, uint64_t seed,
                      int32_t *out_tokens, uint8_t *out_mask, float *out_score,
                      int B, int P, int V, void *stream);
+
+/*
+ * Test hook: caps the number of CTAs the streaming kernel of dd_verify / dd_unmask /
+ * dd_verify_static launches (0 = no cap, one CTA per SM).  Outputs, scores included, are
+ * bit-identical for every cap: which warp computes a (row, chunk) unit never changes the
+ * unit's partial result, and rows are folded from their partials in a fixed order (Eq. 5 and
+ * Eq. 7 are sums over the vocabulary; only the order of their evaluation is at stake).
+ * Process-wide.  Returns DD_OK, or DD_ERR_INVALID_ARG for a negative cap.
+ */
+int dd_debug_set_max_ctas(int max_ctas);
 
 /* Bytes of per-device scratch dd_verify needs for this shape (informational). */
 size_t dd_verify_workspace_bytes(int B, int P, int V);

@@ -23,7 +23,7 @@ DD_LAYOUT_BHND, DD_LAYOUT_BNHD = 0, 1
 EXPORTS = (
     "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_unmask", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
-    "dd_status_string", "dd_last_cuda_error", "dd_version",
+    "dd_status_string", "dd_last_cuda_error", "dd_version", "dd_debug_set_max_ctas",
 )
 
 
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.dd_verify_workspace_bytes.restype = ctypes.c_size_t
         L.dd_launch_count.argtypes = []
         L.dd_launch_count.restype = u64
+        L.dd_debug_set_max_ctas.argtypes = [i32]
+        L.dd_debug_set_max_ctas.restype = i32
         L.dd_status_string.argtypes = [i32]
         L.dd_status_string.restype = ctypes.c_char_p
         L.dd_last_cuda_error.argtypes = []
@@ -226,6 +228,11 @@ def verify_status() -> int:
 
 def launch_count() -> int:
     return int(lib().dd_launch_count())
+
+
+def debug_set_max_ctas(n: int):
+    """Test hook: cap the grid of the streaming verify kernel (0 = no cap)."""
+    _check(lib().dd_debug_set_max_ctas(int(n)))
 
 
 def release():

@@ -10,8 +10,9 @@
 // each logit is read from HBM exactly once.
 //
 // Streaming kernel (V % 8 == 0, 16-byte aligned logits; dd_verify_stream.cuh):
-// persistent CTAs whose warps stream chunks of 8192 logits with the next piece's
-// loads in flight while the current one is computed.
+// persistent CTAs; a producer warp feeds per-warp rings in shared memory with bulk
+// asynchronous copies, consumer warps accumulate chunks of up to 8192 logits from
+// them, a publishing warp counts, folds and decides.
 // Element-wise kernel (any V, any alignment; this file): one CTA of 256 threads
 // per chunk of at most 8192 logits, 2-byte loads with bounds checks.
 //
@@ -25,6 +26,9 @@
 // scratch is ready for the next launch; every fold runs in a fixed order, so the
 // result does not depend on the order in which warps finish.
 #include <stdio.h>
+
+#include <atomic>
+#include <mutex>
 
 #include "dd_verify_stream.cuh"
 
@@ -108,19 +112,20 @@ __device__ __forceinline__ void warp_partial(const uint4 (&rv)[kVecPerThread], c
             for (int h = 0; h < 4; ++h) {
                 const bool ok0 = e0 + 2 * h < n, ok1 = e0 + 2 * h + 1 < n;
                 const float v0 = bf16lo(wv[h]), v1 = bf16hi(wv[h]);
-                if (ok0) s_v0 += ex2_approx(fmaf(v0, kLog2e, -M_v));
-                if (ok1) s_v1 += ex2_approx(fmaf(v1, kLog2e, -M_v));
+                // a logit of -inf is probability zero: no term (also when every logit of the warp is -inf)
+                if (ok0 && v0 != -INFINITY) s_v0 += ex2_approx(fmaf(v0, kLog2e, -M_v));
+                if (ok1 && v1 != -INFINITY) s_v1 += ex2_approx(fmaf(v1, kLog2e, -M_v));
                 if (KL) {
                     const float d0 = bf16lo(wd[h]), d1 = bf16hi(wd[h]);
-                    if (ok0) {
+                    if (ok0 && d0 != -INFINITY) {
                         const float e = ex2_approx(fmaf(d0, kLog2e, -M_d));
                         s_d0 += e;
-                        t0 = fmaf(e, d0 - v0, t0);
+                        if (e > 0.f) t0 = fmaf(e, d0 - v0, t0);      // p_D = 0 contributes no term
                     }
-                    if (ok1) {
+                    if (ok1 && d1 != -INFINITY) {
                         const float e = ex2_approx(fmaf(d1, kLog2e, -M_d));
                         s_d1 += e;
-                        t1 = fmaf(e, d1 - v1, t1);
+                        if (e > 0.f) t1 = fmaf(e, d1 - v1, t1);
                     }
                 }
             }
@@ -178,7 +183,11 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
 // Host side.
 
 // Counters live in their own allocation: it holds nothing else, so it is all zero whenever no
-// launch is in flight, whatever (B, P) the previous call used.
+// launch is in flight, whatever (B, P) the previous call used.  Its last 256 bytes hold the
+// streaming kernel's three words: health, ticket counter, finished CTAs.
+constexpr size_t kControlBytes = 256;
+constexpr size_t kStatusOffset = 0, kTicketOffset = 64, kCtasDoneOffset = 128;
+
 size_t counter_bytes(int B, int P)
 {
     const size_t bp = (size_t)B * P;
@@ -200,32 +209,27 @@ bool streaming_path(const void *drafter, const void *verifier, int V, bool kl)
     return (V % 8 == 0) && (((uintptr_t)verifier & 15) == 0) && (!kl || ((uintptr_t)drafter & 15) == 0);
 }
 
-// Streaming path: pieces per chunk.  Every streaming warp of a CTA takes whole (row, chunk)
-// units in turn, so a CTA's time is rounds * pieces-per-unit; pick the unit size that wastes
-// least for `rows` flagged rows on `ctas` CTAs (a smaller unit only if it saves 5 %), among
-// those whose partials fit `max_partials` (0: no limit).  `even`: only even counts (without a
-// drafter tensor a warp steps through its unit two pieces at a time).
-int pick_pieces(int V, long rows, int ctas, long max_partials, bool even)
+// Streaming path: stages per chunk (a chunk is the work of one warp and yields one partial).
+// Four stages (16 KB of logits) keep the cost of ending a chunk small; fewer when the rows are
+// too few to give every consumer warp of `sms` CTAs a couple of units; more (up to eight) only
+// where the partials would not fit `max_partials` (0: no limit).  The choice depends on the
+// device, never on the grid actually launched.
+int pick_pieces(int V, long rows, int sms, long max_partials, bool kl)
 {
-    int best = kMaxPiecesPerChunk;
-    long best_cost = -1;
-    for (int k = kMaxPiecesPerChunk; k >= kMinPiecesPerChunk; --k) {
-        if (even && (k & 1)) continue;
-        const long nch = (V + (long)k * kPiece - 1) / ((long)k * kPiece);
-        if (max_partials > 0 && rows * nch > max_partials && k != kMaxPiecesPerChunk) continue;
-        const long per_cta = (rows * nch + ctas - 1) / ctas;
-        const long rounds = (per_cta + kSStreamWarps - 1) / kSStreamWarps;
-        const long cost = rounds * k;
-        // a finer cut has more chunk ends: it must save at least 5 % of the pieces
-        if (best_cost < 0 || cost * 20 <= best_cost * 19) { best_cost = cost; best = k; }
-    }
-    return best;
+    const long step = kl ? kPiece : 2 * kPiece;
+    auto chunks_of = [&](int k) { return (V + k * step - 1) / (k * step); };
+    int k = 4;
+    const long want = 2L * kSConsumers * sms;
+    while (k > 1 && rows * chunks_of(k) < want) k >>= 1;
+    const int k_max = kl ? kMaxPiecesPerChunk : kMaxPiecesPerChunk / 2;      // 8192 logits either way
+    while (max_partials > 0 && k < k_max && rows * chunks_of(k) > max_partials) k <<= 1;
+    return k;
 }
 
-void chunking(int V, bool streaming, int pieces, int *nchunks, int *chunk)
+void chunking(int V, bool streaming, bool kl, int pieces, int *nchunks, int *chunk)
 {
     if (streaming) {
-        *chunk = pieces * kPiece;
+        *chunk = pieces * (kl ? kPiece : 2 * kPiece);
         *nchunks = (V + *chunk - 1) / *chunk;
         return;
     }
@@ -236,15 +240,20 @@ void chunking(int V, bool streaming, int pieces, int *nchunks, int *chunk)
     *chunk = c;
 }
 
+std::mutex g_mu;                 // guards the per-device caches below
+int g_sm_count[64] = {};
+bool g_smem_attr_done[64][2] = {};
+std::atomic<int> g_max_ctas{0};  // 0: one CTA per SM; otherwise a cap on the streaming kernel's grid
+
 // Number of SMs of the current device (cached), or a negative status.
 int sm_count_of_current_device()
 {
-    static int cached[64] = {};
     int dev = 0;
     DD_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return dd::cuda_fail(cudaErrorInvalidDevice, "dd_verify: device index");
-    if (!cached[dev]) DD_CUDA_TRY(cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev));
-    return cached[dev];
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_sm_count[dev]) DD_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+    return g_sm_count[dev];
 }
 
 template <bool KL>
@@ -252,9 +261,22 @@ int launch_stream(const VerifyParams &p, cudaStream_t stream)
 {
     const int sms = sm_count_of_current_device();
     if (sms < 0) return sms;
+    int dev = 0;
+    DD_CUDA_TRY(cudaGetDevice(&dev));
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_smem_attr_done[dev][KL ? 1 : 0]) {
+            DD_CUDA_TRY(cudaFuncSetAttribute(verify_stream_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kSRingBytes));
+            g_smem_attr_done[dev][KL ? 1 : 0] = true;
+        }
+    }
     const long units = (long)p.B * p.P * p.nchunks;
-    const long grid = units < sms ? units : sms;
-    verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, 0, stream>>>(p);
+    long grid = (units + kSConsumers - 1) / kSConsumers;
+    if (grid > sms) grid = sms;
+    const int cap = g_max_ctas.load(std::memory_order_relaxed);
+    if (cap > 0 && grid > cap) grid = cap;
+    verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, kSRingBytes, stream>>>(p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
     return DD_OK;
@@ -320,8 +342,8 @@ extern "C" size_t dd_verify_workspace_bytes(int B, int P, int V)
 {
     if (B <= 0 || P <= 0 || V <= 0) return 0;
     int nchunks, chunk;
-    chunking(V, V % 8 == 0, kMinPiecesPerChunk, &nchunks, &chunk);       // the finest cut a launch may choose
-    return workspace_bytes(B, P, nchunks) + counter_bytes(B, P);
+    chunking(V, V % 8 == 0, true, 1, &nchunks, &chunk);       // the finest cut a launch may choose
+    return workspace_bytes(B, P, nchunks) + counter_bytes(B, P) + kControlBytes;
 }
 
 extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits,
@@ -337,27 +359,29 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     const bool streaming = streaming_path(drafter_logits, verifier_logits, V, kl);
 
     VerifyParams p;
-    int pieces = kMaxPiecesPerChunk;
+    int pieces = 4;
     if (streaming) {
         const int sms = sm_count_of_current_device();
         if (sms < 0) return sms;
-        pieces = pick_pieces(V, (long)B * P, sms, (1L << 31) - 1, !kl);
+        pieces = pick_pieces(V, (long)B * P, sms, 0, kl);
     }
-    chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
-    if ((long)B * P * p.nchunks >= (1L << 31)) return DD_ERR_UNSUPPORTED;
+    chunking(V, streaming, kl, pieces, &p.nchunks, &p.chunk);
+    if ((long)B * P * p.nchunks >= (1L << 31) - (1L << 24)) return DD_ERR_UNSUPPORTED;
 
     dd::DeviceCtx *ctx = dd::current_ctx();
     if (!ctx) return DD_ERR_CUDA;
     rc = dd::ensure_bytes(&ctx->verify_ws, &ctx->verify_ws_bytes, workspace_bytes(B, P, p.nchunks));
     if (rc != DD_OK) return rc;
-    // the last 256 bytes of the counter block hold the health word of the streaming kernel
-    rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(B, P) + 256);
+    rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(B, P) + kControlBytes);
     if (rc != DD_OK) return rc;
 
     const size_t bp = (size_t)B * P;
     p.row_counter = (unsigned int *)ctx->verify_cnt;
     p.seq_counter = (unsigned int *)((char *)ctx->verify_cnt + ((bp * 4 + 255) & ~size_t(255)));
-    p.status = (unsigned int *)((char *)ctx->verify_cnt + ctx->verify_cnt_bytes - 256);
+    char *control = (char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes;
+    p.status = (unsigned int *)(control + kStatusOffset);
+    p.ticket = (unsigned int *)(control + kTicketOffset);
+    p.ctas_done = (unsigned int *)(control + kCtasDoneOffset);
     char *w = (char *)ctx->verify_ws;
     p.row_score = (float *)w;          w += (bp * 4 + 255) & ~size_t(255);
     p.row_argmax = (int *)w;           w += (bp * 4 + 255) & ~size_t(255);
@@ -379,21 +403,10 @@ extern "C" int dd_unmask(const void *logits, const int32_t *tokens, const uint8_
                      B, P, V, stream);
 }
 
-extern "C" int dd_verify_status(void)
+extern "C" int dd_debug_set_max_ctas(int max_ctas)
 {
-    dd::DeviceCtx *ctx = dd::current_ctx();
-    if (!ctx) return DD_ERR_CUDA;
-    if (!ctx->verify_cnt) return DD_OK;
-    unsigned int word = 0;
-    DD_CUDA_TRY(cudaDeviceSynchronize());
-    DD_CUDA_TRY(cudaMemcpy(&word, (char *)ctx->verify_cnt + ctx->verify_cnt_bytes - 256, sizeof word,
-                           cudaMemcpyDeviceToHost));
-    if (word != 0) {
-        char text[96];
-        snprintf(text, sizeof text, "verify kernel: bounded wait expired, code 0x%08x", word);
-        dd::set_error_text(text);
-        return DD_ERR_TIMEOUT;
-    }
+    if (max_ctas < 0) return DD_ERR_INVALID_ARG;
+    g_max_ctas.store(max_ctas, std::memory_order_relaxed);
     return DD_OK;
 }
 
@@ -411,17 +424,27 @@ namespace {
 
 constexpr int kStaticMaxRows = 4096;          // B * P
 constexpr int kStaticMaxPartials = 65536;     // B * P * ceil(V / 8192)
-constexpr size_t kStaticCounterBytes = (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255)) +
-                                       (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));   // rows + sequences
-constexpr size_t kStaticRowBytes = 2 * (((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255));  // score + argmax
+constexpr size_t kStaticRowsSlot = ((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255);
+constexpr size_t kStaticCounterBytes = 2 * kStaticRowsSlot + kControlBytes;   // rows, sequences, control words
+constexpr size_t kStaticRowBytes = 2 * kStaticRowsSlot;                       // score + argmax
 constexpr size_t kStaticScratchBytes = kStaticCounterBytes + kStaticRowBytes +
                                        (size_t)kStaticMaxPartials * sizeof(Partial);
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never an address to pass on.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-// Device address of g_static_scratch per device, resolved on the first call made on that device.
+// Device address of g_static_scratch per device, resolved on the first call made on that device
+// (guarded by g_mu).
 unsigned char *g_static_ptr[64] = {};
+
+// The array's address on the current device (null if no call has resolved it yet).
+unsigned char *static_scratch_if_resolved()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mu);
+    return g_static_ptr[dev];
+}
 
 }  // namespace
 
@@ -442,40 +465,72 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     // only chosen where its partials still fit)
     const long coarse_chunks = (V + kSChunk - 1) / kSChunk;
     if ((long)B * P > kStaticMaxRows || (long)B * P * coarse_chunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
-    int pieces = kMaxPiecesPerChunk;
+    int pieces = 4;
     if (streaming) {
         const int sms = sm_count_of_current_device();
         if (sms < 0) return sms;
-        pieces = pick_pieces(V, (long)B * P, sms, kStaticMaxPartials, !kl);
+        pieces = pick_pieces(V, (long)B * P, sms, kStaticMaxPartials, kl);
     }
-    chunking(V, streaming, pieces, &p.nchunks, &p.chunk);
+    chunking(V, streaming, kl, pieces, &p.nchunks, &p.chunk);
     if ((long)B * P * p.nchunks > kStaticMaxPartials) return DD_ERR_UNSUPPORTED;
 
     int dev = -1;
     DD_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return dd::cuda_fail(cudaErrorInvalidDevice, "dd_verify_static: device index");
-    if (!g_static_ptr[dev]) {
-        // set-up, once per device, with that device current
-        void *ptr = nullptr;
-        DD_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
-        g_static_ptr[dev] = static_cast<unsigned char *>(ptr);
+    unsigned char *base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_static_ptr[dev]) {
+            // set-up, once per device, with that device current
+            void *ptr = nullptr;
+            DD_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+            g_static_ptr[dev] = static_cast<unsigned char *>(ptr);
+        }
+        base = g_static_ptr[dev];
     }
-    unsigned char *base = g_static_ptr[dev];
     const size_t bp = (size_t)B * P;
-    const size_t rows_slot = ((size_t)kStaticMaxRows * 4 + 255) & ~size_t(255);
+    unsigned char *control = base + 2 * kStaticRowsSlot;
     p.row_counter = (unsigned int *)base;
-    p.seq_counter = (unsigned int *)(base + rows_slot);
+    p.seq_counter = (unsigned int *)(base + kStaticRowsSlot);
+    p.status = (unsigned int *)(control + kStatusOffset);
+    p.ticket = (unsigned int *)(control + kTicketOffset);
+    p.ctas_done = (unsigned int *)(control + kCtasDoneOffset);
     p.row_score = (float *)(base + kStaticCounterBytes);
-    p.row_argmax = (int *)(base + kStaticCounterBytes + rows_slot);
+    p.row_argmax = (int *)(base + kStaticCounterBytes + kStaticRowsSlot);
     p.partials = (Partial *)(base + kStaticCounterBytes + kStaticRowBytes);
-    p.status = nullptr;
 
     fill_params(p, drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, seed,
                 out_tokens, out_mask, out_score, B, P, V);
 
     cudaStream_t s = (cudaStream_t)stream;
-    // The array keeps whatever the previous call left: the counters must start at zero.
+    // The array keeps whatever the previous call left: the counters must start at zero (the
+    // health word is left alone: it is sticky, like dd_verify's).
     DD_CUDA_TRY(cudaMemsetAsync(p.row_counter, 0, bp * 4, s));
     DD_CUDA_TRY(cudaMemsetAsync(p.seq_counter, 0, (size_t)B * 4, s));
+    DD_CUDA_TRY(cudaMemsetAsync(p.ticket, 0, kControlBytes - kTicketOffset, s));
     return launch(p, streaming, s);
+}
+
+extern "C" int dd_verify_status(void)
+{
+    dd::DeviceCtx *ctx = dd::current_ctx();
+    if (!ctx) return DD_ERR_CUDA;
+    unsigned char *fixed = static_scratch_if_resolved();
+    if (!ctx->verify_cnt && !fixed) return DD_OK;
+    unsigned int word = 0, word_fixed = 0;
+    DD_CUDA_TRY(cudaDeviceSynchronize());
+    if (ctx->verify_cnt)
+        DD_CUDA_TRY(cudaMemcpy(&word, (char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes + kStatusOffset,
+                               sizeof word, cudaMemcpyDeviceToHost));
+    if (fixed)
+        DD_CUDA_TRY(cudaMemcpy(&word_fixed, fixed + 2 * kStaticRowsSlot + kStatusOffset, sizeof word_fixed,
+                               cudaMemcpyDeviceToHost));
+    if (word == 0) word = word_fixed;
+    if (word != 0) {
+        char text[96];
+        snprintf(text, sizeof text, "verify kernel: bounded wait expired, code 0x%08x", word);
+        dd::set_error_text(text);
+        return DD_ERR_TIMEOUT;
+    }
+    return DD_OK;
 }

@@ -21,7 +21,7 @@ constexpr double kLn2 = 0.69314718055994530942;
 struct __align__(16) Partial {   // one per (row, chunk); 32 bytes
     float m_v, s_v;              // verifier: maximum, sum 2^(l*log2e - M) with M = m*log2e rounded once
     int idx;                     // lowest index of the verifier's maximum
-    float m_d;                   // drafter: maximum
+    float m_d;                   // drafter: reference point of its sums (at most its maximum)
     float s_d, t;                // drafter: sum 2^(..), sum 2^(..) (l_D - l_V)
     float pad0, pad1;            // in flight inside a kernel: row and chunk as integer bits
 };
@@ -47,6 +47,8 @@ struct VerifyParams {
     int *row_argmax;             // [B*P]
     Partial *partials;           // [B*P*nchunks]
     unsigned int *status;        // one word: first expired wait of the streaming kernel (may be null)
+    unsigned int *ticket;        // streaming kernel: units drawn beyond the fixed first ones (zero at rest)
+    unsigned int *ctas_done;     // streaming kernel: CTAs that have drawn their last ticket (zero at rest)
 };
 
 __device__ __forceinline__ float ex2_approx(float x)

@@ -1,61 +1,99 @@
 // Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
 //
-// One persistent CTA per SM: fifteen warps stream, one warp publishes.  The flagged rows'
-// (row, chunk) units (3 to 8 pieces of 1024 logits, chosen per launch so that the units of a
-// range come out in whole rounds of the streaming warps) are numbered in row order and cut into equal
-// contiguous ranges, one per CTA (more when a range would not fit the CTA's table).  The
-// range's units go to the streaming warps in turn.  A warp walks its unit in pieces of 1024
-// logits per tensor (2048 of the verifier when there is no drafter tensor): every lane holds
-// four 16-byte vectors per tensor of the current piece (eight of the verifier)
-// in registers and has the loads of the next piece in flight while it computes (the
-// measured copy bandwidth is reached with this depth; a shared-memory ring fed by bulk
-// copies reached it too but cost about four times the instructions per piece).  Within a
-// chunk every lane keeps its own running maxima, reference points and sums (packed bf16x2
-// maxima, packed fp32 pairs); lanes talk to each other only when the chunk ends.  The
-// chunk's partial goes into a table in shared memory; the warp that stores a row's last
-// chunk folds the row there, so a row that lies inside one range costs no global round
-// trip.  Rows cut by a range boundary go through global memory as chunk partials plus one
-// counter update per range.  The publishing warp takes finished rows from a shared-memory
-// queue, stores their scores, updates the sequence counters in batches (one fence per
-// batch) and decides completed sequences, so the streaming warps never wait for global
-// memory other than their logits.
+// One persistent CTA per SM: sixteen consumer warps, one producer warp, one publishing warp.
+//
+// Work.  A flagged row is cut into chunks of a fixed number of logits (a multiple of the stage
+// size); the (row, chunk) units of all flagged rows are numbered in row order.  A unit is the
+// work of one consumer warp and yields one partial.  The first two units of every consumer are
+// fixed by its position in the grid; every further one is drawn from a global ticket counter,
+// one unit ahead of need, so a warp that streams faster simply takes more units.  Which warp
+// computes a unit never changes the unit's partial, and rows are folded from their partials
+// in chunk order, so the results do not depend on the grid or on timing.
+//
+// Data path.  Lane w of the producer warp feeds consumer warp w: it maps the consumer's next
+// unit to its row, and for every stage-sized piece of the unit (1024 logits of both tensors,
+// or 2048 of the verifier alone: 4 KB) issues bulk asynchronous copies from global memory into
+// the consumer's private ring of stages in shared memory, completing on the stage's "full"
+// mbarrier.  The consumer waits for the stage, loads its eight 16-byte vectors per lane, hands
+// the stage back (the "empty" mbarrier) as soon as the first pass has consumed the registers,
+// and accumulates.  Consumers do no address arithmetic and no global loads.
+//
+// Arithmetic.  Within a chunk every lane keeps its own state: packed bf16x2 running maxima of
+// the verifier with the ordinal of the word where each half first rose (the lowest index of
+// the maximum without a second look at the data), and fp32 pair sums S_V, S_D,
+// T = sum 2^(..)(l_D - l_V) against reference points fixed by the lane's first piece of the
+// chunk (any reference works as long as it is reused; an overflow of the range shows up as a
+// non-finite sum and sends the chunk to a careful scalar path, as do logits of -inf).  Lanes
+// talk to each other only when the chunk ends: the 32 lane states become one partial, which
+// goes to the publishing warp through a queue in shared memory.
+//
+// Publication.  The publishing warp stores partials to global memory in batches, counts them
+// per row (one fence per batch), folds the rows it completes in chunk order in fp64 (Eq. 5,
+// Eq. 7), counts rows per sequence and decides the sequences it completes (Section 3.2).
 #pragma once
 
 #include "dd_verify_common.cuh"
 
 namespace ddv {
 
-constexpr int kSStreamWarps = 15;                             // warps that stream
-constexpr int kSWarps = kSStreamWarps + 1;                    // + one that publishes finished chunks
+constexpr int kSConsumers = 16;                               // warps that compute
+constexpr int kSProducerWarp = kSConsumers;                   // one warp that issues the copies
+constexpr int kSPublisherWarp = kSConsumers + 1;              // one warp that publishes partials
+constexpr int kSWarps = kSConsumers + 2;
 constexpr int kSThreads = kSWarps * 32;
-constexpr int kSQueue = 64;                                   // finished-chunk queue slots
-constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per step of a warp
-constexpr int kMinPiecesPerChunk = 3, kMaxPiecesPerChunk = 8; // a (row, chunk) unit is 3072 .. 8192 logits
-constexpr int kSChunk = kPiece * kMaxPiecesPerChunk;
-constexpr int kSTable = 768;                                  // chunk partials a CTA keeps per range
-constexpr unsigned kErrWaitQueue = 0x800;
+constexpr int kSStages = 3;                                   // ring slots per consumer
+constexpr int kSStageBytes = 4096;
+constexpr int kSRingBytes = kSConsumers * kSStages * kSStageBytes;
+constexpr int kSQueue = 64;                                   // finished-unit queue slots
+constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per stage (KL)
+constexpr int kMaxPiecesPerChunk = 8;
+constexpr int kSChunk = kPiece * kMaxPiecesPerChunk;          // coarsest cut of a row: 8192 logits
+constexpr unsigned kErrWaitQueue = 0x800, kErrWaitFull = 0x900, kErrWaitEmpty = 0xA00, kErrWaitUnit = 0xB00;
 
-// Logits per tensor in one step of a warp.  Without a drafter tensor (TRUST, CONF) the registers
-// that would hold the drafter's vectors hold four more vectors of the verifier: the piece is twice
-// as long, so that a warp has as many bytes in flight as in KL mode.
+// Logits per tensor in one stage.  Without a drafter tensor (TRUST, CONF) the half of the stage
+// that would hold the drafter's logits holds 1024 more of the verifier's.
 template <bool KL>
 struct PieceOf {
     static constexpr int value = KL ? kPiece : 2 * kPiece;
 };
 
-__device__ __forceinline__ uint4 ld_stream(const uint4 *ptr)
+// ---- mbarrier and bulk-copy wrappers (shared::cta addresses as 32-bit integers) ----------------
+__device__ __forceinline__ uint32_t s_addr(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ void sbar_init(uint32_t bar, uint32_t count)
 {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(ptr));
-    return r;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void sbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void sbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool sbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bytes (a multiple of 16) from global to shared memory, both 16-byte aligned; completes on `bar`
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // Running state of one lane over the pieces of a chunk.
 struct LaneState {
-    uint32_t max2_v, max2_d;   // packed bf16x2 running maxima (even / odd logits of the lane's words)
-    uint32_t where2_v;         // per half: ordinal of the word that first attained the verifier's maximum
-    float M_v, M_d;            // reference points: lane maximum * log2e
+    uint32_t max2_v;           // packed bf16x2 running maxima of the verifier (even / odd logits of the lane's words)
+    uint32_t where2_v;         // per half: ordinal of the word that first attained that maximum
+    uint32_t max2_d;           // drafter: packed maxima of the lane's first piece (its reference point)
+    float M_v, M_d;            // reference points: maximum of the lane's first piece * log2e
     float2 s_v, s_d, t;        // sums of the even / odd logits
 };
 
@@ -67,19 +105,20 @@ __device__ __forceinline__ void lane_reset(LaneState &L)
     L.s_v = L.s_d = L.t = make_float2(0.f, 0.f);
 }
 
-// One piece (n logits, a multiple of 8; lane's vector j covers logits (lane + 32 j) * 8 ..+7).
-// KL: rv / rd are the verifier's / drafter's vectors 0..3.  Otherwise rv holds the verifier's
-// vectors 0..3 and rd its vectors 4..7.  kFull: no vector is absent.
-template <bool KL, bool kFull>
-__device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecPerThread],
-                                           const uint4 (&rd)[kVecPerThread], int n, int lane, int ordinal)
+// First pass over a piece: the verifier's packed running maxima and where they rose.  Lane's
+// vector j covers logits (lane + 32 j) * 8 ..+7 of the piece.  KL: rv / rd are the verifier's /
+// drafter's vectors 0..3; otherwise rv holds the verifier's vectors 0..3 and rd its vectors 4..7.
+// Absent vectors hold -inf.  `first`: the piece opens a chunk and fixes the lane's reference points.
+template <bool KL>
+__device__ __forceinline__ void lane_pass1(LaneState &L, const uint4 (&rv)[kVecPerThread],
+                                           const uint4 (&rd)[kVecPerThread], int ordinal, bool first)
 {
-    // pass 1: packed running maxima; the word ordinal (within this piece) where a half first rose
-    uint32_t max2_v = L.max2_v, max2_d = L.max2_d, where2 = 0u;
+    uint32_t max2_v = L.max2_v, where2 = 0u;
 #pragma unroll
-    for (int j = 0; j < kVecPerThread; ++j) {
-        const uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
-        const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+    for (int j = 0; j < (KL ? 1 : 2) * kVecPerThread; ++j) {
+        // words are visited in the order of their logits, so a maximum that occurs twice keeps its first place
+        const uint4 &x = j < kVecPerThread ? rv[j] : rd[j - kVecPerThread];
+        const uint32_t wv[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
             const __nv_bfloat162 w = *reinterpret_cast<const __nv_bfloat162 *>(&wv[h]);
@@ -89,29 +128,6 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
             max2_v = *reinterpret_cast<const uint32_t *>(&m_new);
             const uint32_t q2 = (uint32_t)(j * 4 + h) * 0x00010001u;
             where2 = (where2 & ~rose) | (q2 & rose);
-            if (KL) {
-                const __nv_bfloat162 d = *reinterpret_cast<const __nv_bfloat162 *>(&wd[h]);
-                const __nv_bfloat162 md = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&max2_d), d);
-                max2_d = *reinterpret_cast<const uint32_t *>(&md);
-            }
-        }
-    }
-    if (!KL) {
-        // the verifier's vectors 4..7, after 0..3: words are visited in the order of their logits,
-        // so a maximum that occurs twice keeps its first place
-#pragma unroll
-        for (int j = 0; j < kVecPerThread; ++j) {
-            const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-                const __nv_bfloat162 w = *reinterpret_cast<const __nv_bfloat162 *>(&wd[h]);
-                const __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162 *>(&max2_v);
-                const uint32_t rose = __hgt2_mask(w, m);
-                const __nv_bfloat162 m_new = __hmax2(m, w);
-                max2_v = *reinterpret_cast<const uint32_t *>(&m_new);
-                const uint32_t q2 = (uint32_t)((kVecPerThread + j) * 4 + h) * 0x00010001u;
-                where2 = (where2 & ~rose) | (q2 & rose);
-            }
         }
     }
     {
@@ -122,26 +138,35 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
         const uint32_t q2 = where2 + (uint32_t)(ordinal * (KL ? 16 : 32)) * 0x00010001u;
         L.where2_v = (L.where2_v & ~rose) | (q2 & rose);
         L.max2_v = max2_v;
-        L.max2_d = max2_d;
     }
-    // move the reference points; the sums follow
-    const float M_v = fmaxf(bf16lo(max2_v), bf16hi(max2_v)) * kLog2e;
-    {
-        const float f = rescale_factor(L.M_v, M_v);
-        L.s_v = __fmul2_rn(L.s_v, make_float2(f, f));
-        L.M_v = M_v;
+    if (first) {
+        L.M_v = fmaxf(bf16lo(max2_v), bf16hi(max2_v)) * kLog2e;
+        if (KL) {
+            uint32_t max2_d = 0xFF80FF80u;
+#pragma unroll
+            for (int j = 0; j < kVecPerThread; ++j) {
+                const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const __nv_bfloat162 md = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&max2_d),
+                                                      *reinterpret_cast<const __nv_bfloat162 *>(&wd[h]));
+                    max2_d = *reinterpret_cast<const uint32_t *>(&md);
+                }
+            }
+            L.max2_d = max2_d;
+            L.M_d = fmaxf(bf16lo(max2_d), bf16hi(max2_d)) * kLog2e;
+        }
     }
-    float M_d = 0.f;
-    if (KL) {
-        M_d = fmaxf(bf16lo(max2_d), bf16hi(max2_d)) * kLog2e;
-        const float f = rescale_factor(L.M_d, M_d);
-        L.s_d = __fmul2_rn(L.s_d, make_float2(f, f));
-        L.t = __fmul2_rn(L.t, make_float2(f, f));
-        L.M_d = M_d;
-    }
-    // pass 2: one ex2 per logit against the lane's reference
+}
+
+// Second pass: one ex2 per logit against the lane's reference points.  kFull: no vector is absent;
+// otherwise the piece has n logits (a multiple of 8) and vectors beyond them are skipped.
+template <bool KL, bool kFull>
+__device__ __forceinline__ void lane_pass2(LaneState &L, const uint4 (&rv)[kVecPerThread],
+                                           const uint4 (&rd)[kVecPerThread], int n, int lane)
+{
     const float2 log2e2 = make_float2(kLog2e, kLog2e);
-    const float2 nMv2 = make_float2(-M_v, -M_v), nMd2 = make_float2(-M_d, -M_d);
+    const float2 nMv2 = make_float2(-L.M_v, -L.M_v), nMd2 = make_float2(-L.M_d, -L.M_d);
     const float2 neg1 = make_float2(-1.f, -1.f);
     float2 s_v = L.s_v, s_d = L.s_d, t = L.t;
 #pragma unroll
@@ -182,7 +207,8 @@ __device__ __forceinline__ void lane_piece(LaneState &L, const uint4 (&rv)[kVecP
 }
 
 // The chunk has ended: the 32 lane states become one partial (the same bits in every lane):
-// the warp's maxima first, then every lane's sums moved to them and added up.
+// the warp's maxima first, then every lane's sums moved to them and added up.  The drafter's
+// "maximum" is the largest of the lanes' reference points: the sums only need a common one.
 template <bool KL>
 __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chunk_begin, int lane)
 {
@@ -197,10 +223,7 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
     const float my_m = fmaxf(lo_m, hi_m);
     const int my_idx = lo_m > hi_m ? e_lo : (hi_m > lo_m ? e_hi : min(e_lo, e_hi));
     c.m_v = warp_max(my_m);
-    int idx = my_m == c.m_v ? my_idx : 0x7FFFFFFF;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) idx = min(idx, __shfl_xor_sync(0xFFFFFFFFu, idx, o));
-    c.idx = idx;
+    c.idx = __reduce_min_sync(0xFFFFFFFFu, my_m == c.m_v ? my_idx : 0x7FFFFFFF);
     c.s_v = warp_sum((L.s_v.x + L.s_v.y) * rescale_factor(L.M_v, c.m_v * kLog2e));
     c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f;
     if (KL) {
@@ -213,44 +236,90 @@ __device__ __forceinline__ Partial lanes_to_partial(const LaneState &L, int chun
     return c;
 }
 
-// A finished row (or a range's share of a row cut by a range boundary), handed from a
-// streaming warp to the publishing warp.
-struct RowEvent {
-    int row;
-    int whole;        // 1: the row lay inside the range and is folded: score and argmax are final
-    float score;
-    int argmax;
-    int first_slot;   // whole == 0: the range's chunks of this row are table slots first_slot ..
-    int first_chunk;  //             and chunks first_chunk .. of the row,
-    int count;        //             count of them
-    int pad;
+// The same partial computed one logit at a time, straight from global memory, with every special
+// case spelled out: a logit of -inf is probability zero and contributes no term (Eq. 5 runs over
+// the support of p_D), a token only the verifier excludes makes the divergence infinite, and the
+// reference points are the true maxima.  Rare: a chunk comes here only when the packed path
+// produced a non-finite sum.
+template <bool KL>
+__device__ __noinline__ Partial careful_chunk_partial(const uint16_t *verifier_row, const uint16_t *drafter_row,
+                                                      int begin, int end)
+{
+    const int lane = threadIdx.x & 31;
+    float mv = -INFINITY, md = -INFINITY;
+    int idx = 0x7FFFFFFF;
+    for (int e = begin + lane; e < end; e += 32) {
+        const float v = bf16lo((uint32_t)verifier_row[e]);
+        if (v > mv) { mv = v; idx = e; }
+        if (KL) md = fmaxf(md, bf16lo((uint32_t)drafter_row[e]));
+    }
+    Partial c;
+    c.m_v = warp_max(mv);
+    c.idx = __reduce_min_sync(0xFFFFFFFFu, (mv == c.m_v && idx != 0x7FFFFFFF) ? idx : 0x7FFFFFFF);
+    if (c.idx == 0x7FFFFFFF) c.idx = begin;               // every logit is -inf: the lowest index
+    c.m_d = KL ? warp_max(md) : 0.f;
+    const float Mv = c.m_v * kLog2e, Md = c.m_d * kLog2e;
+    float sv = 0.f, sd = 0.f, t = 0.f;
+    for (int e = begin + lane; e < end; e += 32) {
+        const float v = bf16lo((uint32_t)verifier_row[e]);
+        if (v != -INFINITY) sv += ex2_approx(fmaf(v, kLog2e, -Mv));
+        if (KL) {
+            const float d = bf16lo((uint32_t)drafter_row[e]);
+            if (d != -INFINITY) {
+                const float ed = ex2_approx(fmaf(d, kLog2e, -Md));
+                sd += ed;
+                if (ed > 0.f) t = fmaf(ed, d - v, t);
+            }
+        }
+    }
+    c.s_v = warp_sum(sv);
+    c.s_d = KL ? warp_sum(sd) : 0.f;
+    c.t = KL ? warp_sum(t) : 0.f;
+    c.pad0 = c.pad1 = 0.f;
+    return c;
+}
+
+// A finished (row, chunk) unit, handed from a consumer warp to the publishing warp.
+struct __align__(16) UnitEvent {
+    int row, chunk, pad0, pad1;
+    Partial part;
 };
 
-// Queue of row events between the streaming warps (many producers) and the publishing warp
+// Queue of unit events between the consumer warps (many producers) and the publishing warp
 // (one consumer), in shared memory.
 struct EventQueue {
-    RowEvent entry[kSQueue];
+    UnitEvent entry[kSQueue];
     unsigned int ready[kSQueue];     // sequence number + 1 of the entry the slot holds
     unsigned int tail;               // next sequence number to hand out
     unsigned int head;               // entries below this have been taken
-    unsigned int done;               // streaming warps that have finished the current range
+    unsigned int done;               // consumer warps that have finished
     unsigned int pad;
 };
 
-// One lane of a streaming warp hands over an entry.  False if the queue stayed full.
-__device__ __forceinline__ bool queue_push(EventQueue &q, const RowEvent &e)
+// A consumer warp hands over a unit (every lane holds the same partial).  False if the queue
+// stayed full.
+__device__ __forceinline__ bool queue_push(EventQueue &q, int row, int chunk, const Partial &part, int lane)
 {
-    const unsigned int seq = atomicAdd(&q.tail, 1u);
-    volatile unsigned int *head = &q.head;
-    unsigned it = 0;
-    while (seq - *head >= (unsigned)kSQueue) {
-        if (++it > (1u << 22)) return false;
-        __nanosleep(64);
+    int ok = 1;
+    if (lane == 0) {
+        const unsigned int seq = atomicAdd(&q.tail, 1u);
+        volatile unsigned int *head = &q.head;
+        unsigned it = 0;
+        while (seq - *head >= (unsigned)kSQueue) {
+            if (++it > (1u << 22)) { ok = 0; break; }
+            __nanosleep(64);
+        }
+        if (ok) {
+            UnitEvent *e = &q.entry[seq % kSQueue];
+            float4 *dst = reinterpret_cast<float4 *>(e);
+            dst[0] = make_float4(__int_as_float(row), __int_as_float(chunk), 0.f, 0.f);
+            dst[1] = make_float4(part.m_v, part.s_v, __int_as_float(part.idx), part.m_d);
+            dst[2] = make_float4(part.s_d, part.t, 0.f, 0.f);
+            __threadfence_block();
+            *(volatile unsigned int *)&q.ready[seq % kSQueue] = seq + 1u;
+        }
     }
-    q.entry[seq % kSQueue] = e;
-    __threadfence_block();
-    *(volatile unsigned int *)&q.ready[seq % kSQueue] = seq + 1u;
-    return true;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
 }  // namespace ddv

@@ -40,16 +40,21 @@ __device__ __forceinline__ void rows_done(const VerifyParams &p, SeqTally &tally
 template <bool KL>
 __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const VerifyParams p)
 {
-    __shared__ __align__(16) Partial s_table[kSTable];          // chunk partials of the current range
-    __shared__ int s_rows[kSTable + 2];                          // flagged rows the range touches
-    __shared__ unsigned int s_rowcnt[kSTable + 2];               // their chunks stored so far
+    extern __shared__ __align__(128) unsigned char s_ring[];     // [consumer][stage][kSStageBytes]
+    __shared__ __align__(8) unsigned long long s_full[kSConsumers][kSStages];    // mbarriers: the stage holds data
+    __shared__ __align__(8) unsigned long long s_empty[kSConsumers][kSStages];   // mbarriers: the stage is free
+    __shared__ __align__(16) int4 s_meta[kSConsumers][kSStages];  // what the stage holds
+    __shared__ __align__(8) unsigned long long s_mailbox[kSConsumers][2];       // (unit index + 1) << 32 | ticket
     __shared__ __align__(16) EventQueue s_queue;
+    __shared__ int s_prefix[kSThreads + 1];                       // flagged rows before each thread's slice
     __shared__ int s_scan[kSWarps];
+    __shared__ int s_abort;                                       // a bounded wait expired somewhere in the CTA
     __shared__ DecideStage s_decide;                              // decision stage (publishing warp only)
 
     const unsigned full = 0xFFFFFFFFu;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nch = p.nchunks;
+    constexpr int kStep = PieceOf<KL>::value;                    // logits per stage
 
     // ---- every thread counts the flagged rows of its contiguous slice of the B*P rows; the block
     // scan gives each thread the number of flagged rows before its slice, and the total
@@ -58,7 +63,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     const long my_begin = min(n_rows, (long)tid * slice), my_end = min(n_rows, my_begin + slice);
     int my_count = 0;
     for (long r = my_begin; r < my_end; ++r) my_count += p.flags[r] != 0;
-    long my_prefix, total_flagged;
+    long total_flagged;
     {
         int incl = my_count;
 #pragma unroll
@@ -67,6 +72,19 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             if (lane >= o) incl += v;
         }
         if (lane == 31) s_scan[warp] = incl;
+        if (tid < kSQueue) s_queue.ready[tid] = 0u;
+        if (tid == 0) {
+            s_queue.tail = s_queue.head = s_queue.done = 0u;
+            s_abort = 0;
+            for (int w = 0; w < kSConsumers; ++w) {
+                for (int s = 0; s < kSStages; ++s) {
+                    sbar_init(s_addr(&s_full[w][s]), 1);
+                    sbar_init(s_addr(&s_empty[w][s]), 1);
+                }
+                s_mailbox[w][0] = s_mailbox[w][1] = 0ull;
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
         __syncthreads();
         int before = 0, all = 0;
         for (int w = 0; w < kSWarps; ++w) {
@@ -74,276 +92,306 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             if (w < warp) before += v;
             all += v;
         }
-        my_prefix = (long)before + incl - my_count;
+        s_prefix[tid] = before + incl - my_count;
+        if (tid == 0) s_prefix[kSThreads] = all;
         total_flagged = all;
     }
+    __syncthreads();
     const long total_units = total_flagged * nch;
-    // equal ranges, each small enough for the table, their number a multiple of the CTAs
-    const long per_cta = (total_units + gridDim.x - 1) / gridDim.x;
-    const long rounds = per_cta > kSTable ? (per_cta + kSTable - 1) / kSTable : 1;
-    const long n_ranges = rounds * gridDim.x;
+    volatile int *abort_flag = &s_abort;
 
-    SeqTally tally;
-    tally.b = -1;
-    tally.target = 0;
-    __shared__ float s_rehearsal[2];
-    // sequences without a single flagged row pass through; this CTA's share of them
-    auto pass_through = [&]() {
-        for (int b = blockIdx.x; b < p.B; b += gridDim.x)
-            if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
-    };
-    bool rehearsed = false;
-    bool queue_ok = true;
-
-    for (long range = blockIdx.x; range < n_ranges; range += gridDim.x) {
-        const long lo = total_units * range / n_ranges, hi = total_units * (range + 1) / n_ranges;
-        if (hi <= lo) continue;                                   // uniform over the CTA
-        const int n_units = (int)(hi - lo);
-        const long f_lo = lo / nch, f_hi = (hi - 1) / nch;        // flagged-row ordinals the range touches
-
-        __syncthreads();                                          // the previous range is fully drained
-        {
-            long ord = my_prefix;
-            for (long r = my_begin; r < my_end && ord <= f_hi; ++r) {
-                if (p.flags[r]) {
-                    if (ord >= f_lo) s_rows[ord - f_lo] = (int)r;
-                    ++ord;
-                }
-            }
-            for (int i = tid; i < (int)(f_hi - f_lo + 1); i += kSThreads) s_rowcnt[i] = 0u;
-            if (tid < kSQueue) s_queue.ready[tid] = 0u;
-            if (tid == 0) {
-                s_queue.tail = s_queue.head = s_queue.done = 0u;
-            }
-        }
-        __syncthreads();
-
-        if (warp == kSStreamWarps) {
-            // =============================================================== publishing warp
-            if (!rehearsed) {
-                // nothing is finished yet: bring the code of the row fold and of the decision stage
-                // into the instruction caches now, not at the end of the launch
-                rehearsed = true;
-                float sc;
-                int am;
-                Partial *fake = reinterpret_cast<Partial *>(s_decide.key);      // free until a sequence ends
-                {
-                    Partial f;
-                    f.m_v = 1.f + lane; f.s_v = 1.5f; f.idx = lane; f.m_d = 0.5f * lane; f.s_d = 1.25f; f.t = 0.125f;
-                    f.pad0 = f.pad1 = 0.f;
-                    fake[lane] = f;
-                }
-                __syncwarp();
-                fold_partials<KL>(fake, 32, sc, am);
-                if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
-                decide_sequence_rehearsal(p, &s_decide);
-                pass_through();
-            }
-            {
-                // the sequence this range ends in: its size is needed when its rows are counted
-                const int b_last = s_rows[(int)(f_hi - f_lo)] / p.P;
-                if (tally.b != b_last) {
-                    tally.b = b_last;
-                    tally.target = count_flagged(p, b_last);
-                }
-            }
-            unsigned int head = 0;
-            for (unsigned idle = 0;;) {
-                const unsigned int mine = head + lane;
-                const bool ready = *(volatile unsigned int *)&s_queue.ready[mine % kSQueue] == mine + 1u;
-                const unsigned mask = __ballot_sync(full, ready);
-                const int n = mask == full ? 32 : __ffs(~mask) - 1;      // contiguous ready entries
-                if (n == 0) {
-                    const unsigned int done = *(volatile unsigned int *)&s_queue.done;
-                    const unsigned int tail = *(volatile unsigned int *)&s_queue.tail;
-                    if (done == (unsigned)kSStreamWarps && tail == head) break;
-                    if (++idle > (1u << 24)) {     // the streaming warps never finished
-                        if (lane == 0 && p.status) atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
-                        break;
-                    }
-                    __nanosleep(250);
-                    continue;
-                }
-                idle = 0;
-                __threadfence_block();
-                RowEvent e = s_queue.entry[(lane < n ? mine : head) % kSQueue];
-                __syncwarp();
-                head += n;
-                if (lane == 0) *(volatile unsigned int *)&s_queue.head = head;
-                const bool mine_ok = lane < n;
-
-                // rows cut by a range boundary: this range's chunk partials go to global memory
-                unsigned parts = __ballot_sync(full, mine_ok && !e.whole);
-                for (unsigned m = parts; m; m &= m - 1) {
-                    const int src = __ffs(m) - 1;
-                    const int row = __shfl_sync(full, e.row, src), slot0 = __shfl_sync(full, e.first_slot, src);
-                    const int chunk0 = __shfl_sync(full, e.first_chunk, src), cnt = __shfl_sync(full, e.count, src);
-                    Partial *dst = p.partials + (size_t)row * nch + chunk0;
-                    for (int i = lane; i < 2 * cnt; i += 32)
-                        __stcg(reinterpret_cast<float4 *>(dst) + i, reinterpret_cast<const float4 *>(s_table + slot0)[i]);
-                }
-                if (parts) {
-                    __threadfence();
-                    bool complete = false;
-                    if (mine_ok && !e.whole)
-                        complete = atomicAdd(p.row_counter + e.row, (unsigned)e.count) + (unsigned)e.count == (unsigned)nch;
-                    unsigned fold = __ballot_sync(full, complete);
-                    if (fold) __threadfence();
-                    for (unsigned m = fold; m; m &= m - 1) {
-                        const int src = __ffs(m) - 1;
-                        const int row = __shfl_sync(full, e.row, src);
-                        float score;
-                        int argmax;
-                        fold_partials<KL>(p.partials + (size_t)row * nch, nch, score, argmax);
-                        if (lane == src) {
-                            e.whole = 1;
-                            e.score = score;
-                            e.argmax = argmax;
-                            p.row_counter[row] = 0u;      // ready for the next launch
-                        }
-                    }
-                }
-                // finished rows: store, fence once, count them per sequence
-                const bool finished = mine_ok && e.whole;
-                if (finished) {
-                    __stcg(p.row_score + e.row, e.score);
-                    __stcg(p.row_argmax + e.row, e.argmax);
-                }
-                unsigned fin = __ballot_sync(full, finished);
-                if (fin) __threadfence();
-                while (fin) {
-                    const int src = __ffs(fin) - 1;
-                    const int b = __shfl_sync(full, e.row, src) / p.P;
-                    const unsigned same = __ballot_sync(full, finished && e.row / p.P == b) & fin;
-                    fin &= ~same;
-                    rows_done(p, tally, b, __popc(same), &s_decide);
-                }
-            }
-            continue;       // next range
-        }
-
-        // =================================================================== streaming warps
-        const unsigned ulo = (unsigned)lo, uhi = (unsigned)hi, uflo = (unsigned)f_lo;   // units fit 31 bits
-        constexpr int kStep = PieceOf<KL>::value;                                        // logits per piece
-        const int chunk_len = p.chunk, chunk_pieces = p.chunk / kStep;                  // logits, pieces per chunk
-        const int last_pieces = (p.V - (nch - 1) * chunk_len + kStep - 1) / kStep;         // of a row's last chunk
-
-        // Units of the range go to the streaming warps in turn: warp w takes units w, w + 15, ...
-        // A cursor walks one warp's pieces in order (all lanes hold the same values).
-        struct Cursor {
-            int t;              // unit within the range (= its table slot); >= n_units: past the end
-            int local_row;      // the unit's row, numbered within the range
-            int chunk, piece, npieces, row;
-        };
-        auto enter_unit = [&](Cursor &c) {
-            if (c.t >= n_units) return;
-            c.npieces = c.chunk == nch - 1 ? last_pieces : chunk_pieces;
-            c.row = s_rows[c.local_row];
-        };
-        auto advance = [&](Cursor &c) {
-            if (++c.piece < c.npieces) return;
-            c.piece = 0;
-            c.t += kSStreamWarps;
-            c.chunk += kSStreamWarps;
-            if (c.chunk >= nch) {
-                const int q = c.chunk / nch;
-                c.chunk -= q * nch;
-                c.local_row += q;
-            }
-            enter_unit(c);
-        };
-        // the lane's vectors of the cursor's piece, -inf where the row has ended: four per tensor, or
-        // (no drafter tensor) eight of the verifier, the second four in d
-        auto fetch = [&](const Cursor &c, uint4 (&v)[kVecPerThread], uint4 (&d)[kVecPerThread]) {
-            const int e_begin = c.chunk * chunk_len + c.piece * kStep;
-            const int n = p.V - e_begin;                      // logits left in the row
-            const size_t off = (size_t)c.row * p.V + e_begin;
-            const uint4 *gv = reinterpret_cast<const uint4 *>(p.verifier + off) + lane;
-            const uint4 *gd = KL ? reinterpret_cast<const uint4 *>(p.drafter + off) + lane : gv + 32 * kVecPerThread;
-            if (n >= kStep) {
-#pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) {
-                    v[j] = ld_stream(gv + 32 * j);
-                    d[j] = ld_stream(gd + 32 * j);
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) {
-                    v[j] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-                    d[j] = v[j];
-                    if ((lane + 32 * j) * 8 < n) v[j] = ld_stream(gv + 32 * j);
-                    if ((lane + 32 * (KL ? j : kVecPerThread + j)) * 8 < n) d[j] = ld_stream(gd + 32 * j);
-                }
-            }
-        };
-
-        Cursor cc;
-        {
-            cc.t = warp;
-            cc.piece = 0; cc.npieces = 0; cc.row = 0;
-            const unsigned unit = ulo + (unsigned)warp, f = unit / (unsigned)nch;
-            cc.chunk = (int)(unit - f * (unsigned)nch);
-            cc.local_row = (int)(f - uflo);
-            enter_unit(cc);
-        }
-        Cursor nc = cc;                                       // the piece whose loads are in flight
-        uint4 nv[kVecPerThread], nd[kVecPerThread];
-        if (nc.t < n_units) fetch(nc, nv, nd);
-
+    if (warp < kSConsumers) {
+        // ===================================================================== consumer warps
+        const uint32_t ring = s_addr(s_ring) + (uint32_t)(warp * kSStages * kSStageBytes);
+        const unsigned char *ring_gen = s_ring + warp * kSStages * kSStageBytes;
+        unsigned int ticket = 0;          // lane 0: drawn at the start of unit j for unit j + 2
+        unsigned units = 0;               // units started
+        unsigned err = 0;
         LaneState L;
         lane_reset(L);
-        while (cc.t < n_units) {
-            uint4 rv[kVecPerThread], rd[kVecPerThread];
-#pragma unroll
-            for (int j = 0; j < kVecPerThread; ++j) { rv[j] = nv[j]; rd[j] = nd[j]; }
-            advance(nc);
-            if (nc.t < n_units) fetch(nc, nv, nd);            // in flight while this piece is computed
-
-            const int n = min(kStep, p.V - (cc.chunk * chunk_len + cc.piece * kStep));
-            if (n == kStep) lane_piece<KL, true>(L, rv, rd, n, lane, cc.piece);
-            else lane_piece<KL, false>(L, rv, rd, n, lane, cc.piece);
-            const bool chunk_ends = cc.piece == cc.npieces - 1;
-            const Cursor done = cc;
-            advance(cc);
-            if (!chunk_ends) continue;
-
-            // ---- the chunk is complete: into the table; the warp that completes the range's share
-            // of a row hands the row on
-            const Partial part = lanes_to_partial<KL>(L, done.chunk * chunk_len, lane);
-            lane_reset(L);
-            const unsigned row_first = (uflo + (unsigned)done.local_row) * (unsigned)nch;   // the row's unit 0
-            const unsigned first_unit = max(ulo, row_first), end_unit = min(uhi, row_first + (unsigned)nch);
-            const int share = (int)(end_unit - first_unit);
-            int complete = 0;
-            if (lane == 0) {
-                s_table[done.t] = part;
-                __threadfence_block();
-                complete = atomicAdd(&s_rowcnt[done.local_row], 1u) + 1u == (unsigned)share;
+        for (unsigned it = 0;; ++it) {
+            const unsigned stage = it % kSStages, use = it / kSStages;
+            {
+                const uint32_t bar = s_addr(&s_full[warp][stage]);
+                bool arrived = false;
+                for (unsigned spin = 0; spin < (1u << 22); ++spin) {
+                    if (sbar_try_wait(bar, use & 1)) { arrived = true; break; }
+                    if (spin > 32) {
+                        __nanosleep(64);
+                        if (*abort_flag) break;
+                    }
+                }
+                if (!arrived) { err = kErrWaitFull; break; }
             }
-            complete = __shfl_sync(full, complete, 0);
-            if (!complete) continue;
-            __threadfence_block();
-            RowEvent e;
-            e.row = done.row;
-            e.whole = share == nch;
-            e.score = 0.f;
-            e.argmax = 0;
-            e.first_slot = (int)(first_unit - ulo);
-            e.first_chunk = (int)(first_unit - row_first);
-            e.count = share;
-            e.pad = 0;
-            if (e.whole) fold_partials<KL>(s_table + e.first_slot, nch, e.score, e.argmax);
-            if (lane == 0) queue_ok &= queue_push(s_queue, e);
+            const int4 meta = s_meta[warp][stage];            // n logits, flags | piece << 8, row, chunk
+            const int n = meta.x;
+            if (n == 0) break;                                // no more units for this warp
+            const bool first = (meta.y & 1) != 0, last = (meta.y & 2) != 0;
+            if (first) {
+                if (lane == 0) {
+                    // the unit after this one becomes known to the producer; the one after that is drawn
+                    if (units >= 1)
+                        *(volatile unsigned long long *)&s_mailbox[warp][(units + 1) & 1] =
+                            ((unsigned long long)(units + 2) << 32) | ticket;
+                    ticket = atomicAdd(p.ticket, 1u);
+                }
+                ++units;
+            }
+            uint4 rv[kVecPerThread], rd[kVecPerThread];
+            {
+                const uint4 *sv = reinterpret_cast<const uint4 *>(ring_gen + stage * kSStageBytes) + lane;
+                const uint4 *sd = sv + (kSStageBytes / 2) / 16;
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    rv[j] = sv[32 * j];
+                    rd[j] = sd[32 * j];
+                }
+                if (n < kStep) {
+                    // what lies beyond the row's end in the stage is stale: -inf instead
+                    const uint4 ninf = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        if ((lane + 32 * j) * 8 >= n) rv[j] = ninf;
+                        if ((lane + 32 * (KL ? j : kVecPerThread + j)) * 8 >= n) rd[j] = ninf;
+                    }
+                }
+            }
+            lane_pass1<KL>(L, rv, rd, meta.y >> 8, first);
+            // every lane's vectors are in registers (the first pass has used them): the stage goes back
+            __syncwarp();
+            if (lane == 0) sbar_arrive(s_addr(&s_empty[warp][stage]));
+            if (n == kStep) lane_pass2<KL, true>(L, rv, rd, n, lane);
+            else lane_pass2<KL, false>(L, rv, rd, n, lane);
+            if (!last) continue;
+
+            // ---- the chunk is complete: one partial, handed to the publishing warp
+            Partial part = lanes_to_partial<KL>(L, meta.w * p.chunk, lane);
+            lane_reset(L);
+            if (!(isfinite(part.s_v) && isfinite(part.s_d) && isfinite(part.t) && part.m_v > -INFINITY)) {
+                const int begin = meta.w * p.chunk;
+                part = careful_chunk_partial<KL>(p.verifier + (size_t)meta.z * p.V,
+                                                 KL ? p.drafter + (size_t)meta.z * p.V : nullptr,
+                                                 begin, min(p.V, begin + p.chunk));
+            }
+            if (!queue_push(s_queue, meta.z, meta.w, part, lane)) { err = kErrWaitQueue; break; }
         }
         if (lane == 0) {
+            if (err) {
+                *abort_flag = 1;
+                if (p.status) atomicCAS(p.status, 0u, err | (blockIdx.x & 0xFF));
+            }
             __threadfence_block();
             atomicAdd(&s_queue.done, 1u);
         }
+    } else if (warp == kSProducerWarp) {
+        // ===================================================================== producer warp
+        // lane w feeds consumer w; lanes poll in lockstep and never block on one consumer
+        const int w = lane;
+        enum { kNeed, kHave, kLast, kDone };
+        int state = w < kSConsumers ? kNeed : kDone;
+        unsigned it = 0;                  // stages issued to this consumer
+        unsigned k = 0;                   // units taken for this consumer
+        int row = 0, chunk = 0, piece = 0, npieces = 0;
+        unsigned stuck = 0;
+        const long static0 = (long)blockIdx.x * kSConsumers + w;
+        const long static1 = (long)gridDim.x * kSConsumers + static0;
+        const long ticket_base = 2L * gridDim.x * kSConsumers;
+        const int chunk_pieces = p.chunk / kStep;
+        const int last_pieces = (p.V - (nch - 1) * p.chunk + kStep - 1) / kStep;         // of a row's last chunk
+        const uint32_t ring = s_addr(s_ring) + (uint32_t)(w * kSStages * kSStageBytes);
+        while (__any_sync(full, state != kDone)) {
+            bool progress = false;
+            if (state == kNeed) {
+                long unit = -2;                                   // -2: not known yet
+                if (k == 0) unit = static0;
+                else if (k == 1) unit = static1;
+                else {
+                    const unsigned long long m = *(volatile unsigned long long *)&s_mailbox[w][k & 1];
+                    if ((unsigned)(m >> 32) == k + 1u) unit = ticket_base + (long)(unsigned)m;
+                }
+                if (unit != -2) {
+                    if (unit >= total_units) {
+                        state = kLast;
+                    } else {
+                        const int f = (int)(unit / nch);          // ordinal of the flagged row
+                        chunk = (int)(unit - (long)f * nch);
+                        // the thread slice that holds flagged row f, then the row within it
+                        int lo = 0, hi = kSThreads - 1;
+                        while (lo < hi) {
+                            const int mid = (lo + hi + 1) >> 1;
+                            if (s_prefix[mid] <= f) lo = mid; else hi = mid - 1;
+                        }
+                        long r = (long)lo * slice;
+                        const long r_end = min(n_rows, r + slice);
+                        int ord = s_prefix[lo];
+                        for (; r < r_end; ++r) {
+                            if (p.flags[r]) {
+                                if (ord == f) break;
+                                ++ord;
+                            }
+                        }
+                        row = (int)r;
+                        npieces = chunk == nch - 1 ? last_pieces : chunk_pieces;
+                        piece = 0;
+                        state = kHave;
+                    }
+                    ++k;
+                    progress = true;
+                }
+            }
+            if (state == kHave || state == kLast) {
+                const unsigned stage = it % kSStages, use = it / kSStages;
+                if (use == 0 || sbar_try_wait(s_addr(&s_empty[w][stage]), (use - 1) & 1)) {
+                    const uint32_t bar = s_addr(&s_full[w][stage]);
+                    if (state == kLast) {
+                        s_meta[w][stage] = make_int4(0, 0, 0, 0);
+                        sbar_arrive(bar);
+                        state = kDone;
+                    } else {
+                        const int e_begin = chunk * p.chunk + piece * kStep;
+                        const int n = min(kStep, p.V - e_begin);
+                        const int fl = (piece == 0 ? 1 : 0) | (piece == npieces - 1 ? 2 : 0) | (piece << 8);
+                        s_meta[w][stage] = make_int4(n, fl, row, chunk);
+                        const uint32_t bytes = (uint32_t)n * 2u;
+                        const uint32_t dst = ring + stage * kSStageBytes;
+                        const size_t off = (size_t)row * p.V + e_begin;
+                        sbar_expect_tx(bar, KL ? 2u * bytes : bytes);
+                        bulk_load(dst, p.verifier + off, bytes, bar);
+                        if (KL) bulk_load(dst + kSStageBytes / 2, p.drafter + off, bytes, bar);
+                        if (++piece == npieces) state = kNeed;
+                    }
+                    ++it;
+                    progress = true;
+                }
+            }
+            if (progress) {
+                stuck = 0;
+            } else if (state != kDone && ++stuck > (1u << 21)) {
+                // the consumer never freed a stage or never named its next unit
+                *abort_flag = 1;
+                if (p.status) atomicCAS(p.status, 0u, (state == kNeed ? kErrWaitUnit : kErrWaitEmpty) | (blockIdx.x & 0xFF));
+                state = kDone;
+            }
+            if (*abort_flag) break;
+            if (!__any_sync(full, progress)) __nanosleep(100);
+        }
+    } else {
+        // ===================================================================== publishing warp
+        SeqTally tally;
+        tally.b = -1;
+        tally.target = 0;
+        {
+            // nothing is finished yet: bring the code of the row fold and of the decision stage
+            // into the instruction caches now, not at the end of the launch
+            __shared__ float s_rehearsal[2];
+            float sc;
+            int am;
+            Partial *fake = reinterpret_cast<Partial *>(s_decide.key);      // free until a sequence ends
+            {
+                Partial f;
+                f.m_v = 1.f + lane; f.s_v = 1.5f; f.idx = lane; f.m_d = 0.5f * lane; f.s_d = 1.25f; f.t = 0.125f;
+                f.pad0 = f.pad1 = 0.f;
+                fake[lane] = f;
+            }
+            __syncwarp();
+            fold_partials<KL>(fake, 32, sc, am);
+            if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
+            decide_sequence_rehearsal(p, &s_decide);
+            // sequences without a single flagged row pass through; this CTA's share of them
+            for (int b = blockIdx.x; b < p.B; b += gridDim.x)
+                if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
+        }
+        unsigned int head = 0;
+        for (unsigned idle = 0;;) {
+            const unsigned int mine = head + lane;
+            const bool ready = *(volatile unsigned int *)&s_queue.ready[mine % kSQueue] == mine + 1u;
+            const unsigned mask = __ballot_sync(full, ready);
+            const int n = mask == full ? 32 : __ffs(~mask) - 1;      // contiguous ready entries
+            if (n == 0) {
+                const unsigned int done = *(volatile unsigned int *)&s_queue.done;
+                const unsigned int tail = *(volatile unsigned int *)&s_queue.tail;
+                if (done == (unsigned)kSConsumers && tail == head) break;
+                if (++idle > (1u << 23)) {     // the consumer warps never finished
+                    if (lane == 0) {
+                        *abort_flag = 1;
+                        if (p.status) atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
+                    }
+                    break;
+                }
+                __nanosleep(200);
+                continue;
+            }
+            idle = 0;
+            __threadfence_block();
+            const bool mine_ok = lane < n;
+            const UnitEvent *src = &s_queue.entry[(mine_ok ? mine : head) % kSQueue];
+            const float4 e0 = reinterpret_cast<const float4 *>(src)[0];
+            const float4 e1 = reinterpret_cast<const float4 *>(src)[1];
+            const float4 e2 = reinterpret_cast<const float4 *>(src)[2];
+            const int row = __float_as_int(e0.x), chunk = __float_as_int(e0.y);
+            __syncwarp();
+            head += n;
+            if (lane == 0) *(volatile unsigned int *)&s_queue.head = head;
+
+            // the partials go to global memory; one fence for the batch, then one count per unit
+            if (mine_ok) {
+                float4 *dst = reinterpret_cast<float4 *>(p.partials + (size_t)row * nch + chunk);
+                __stcg(dst, e1);
+                __stcg(dst + 1, e2);
+            }
+            __threadfence();
+            bool complete = false;
+            if (mine_ok) complete = atomicAdd(p.row_counter + row, 1u) + 1u == (unsigned)nch;
+            const unsigned fold = __ballot_sync(full, complete);
+            if (fold == 0u) continue;
+            __threadfence();
+            float my_score = 0.f;
+            int my_argmax = 0;
+            for (unsigned m = fold; m; m &= m - 1) {
+                const int from = __ffs(m) - 1;
+                const int r = __shfl_sync(full, row, from);
+                float score;
+                int argmax;
+                fold_partials<KL>(p.partials + (size_t)r * nch, nch, score, argmax);
+                if (lane == from) {
+                    my_score = score;
+                    my_argmax = argmax;
+                    p.row_counter[r] = 0u;      // ready for the next launch
+                }
+            }
+            // finished rows: store, fence once, count them per sequence
+            if (complete) {
+                __stcg(p.row_score + row, my_score);
+                __stcg(p.row_argmax + row, my_argmax);
+            }
+            __threadfence();
+            unsigned fin = fold;
+            while (fin) {
+                const int from = __ffs(fin) - 1;
+                const int b = __shfl_sync(full, row, from) / p.P;
+                const unsigned same = __ballot_sync(full, complete && row / p.P == b) & fin;
+                fin &= ~same;
+                rows_done(p, tally, b, __popc(same), &s_decide);
+            }
+        }
     }
 
-    if (warp == kSStreamWarps && !rehearsed) pass_through();      // this CTA had no range
-    if (warp < kSStreamWarps && !queue_ok && lane == 0 && p.status)
-        atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
+    // ---- the ticket counter goes back to zero once every CTA has drawn its last ticket
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait expired: give copies that may still be in flight time to land before the shared
+        // memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(p.ctas_done, 1u) == gridDim.x - 1) {
+            *p.ticket = 0u;
+            __threadfence();
+            *p.ctas_done = 0u;
+        }
+    }
 }
 
 }  // namespace ddv

@@ -217,3 +217,53 @@ def test_scratch_survives_changing_shapes(dd, oracle_mod):
     for n, (B, P, V) in enumerate(shapes):
         dra, ver, tokens, flags = synth.verify_inputs(B, P, V, max(1, P // 2), 0.2, seed=100 + n)
         compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 3, n)
+
+
+@pytest.fixture
+def cta_cap(dd):
+    """Caps the streaming kernel's grid for one test and lifts the cap afterwards."""
+    yield dd.debug_set_max_ctas
+    dd.debug_set_max_ctas(0)
+
+
+def test_results_do_not_depend_on_the_grid(dd, oracle_mod, cta_cap):
+    """Same inputs on 1, 7, 37 CTAs and on every SM: tokens, masks and scores bit-identical (which
+    warp computes a unit, and in which order units finish, must not matter)."""
+    cases = [
+        (synth.verify_config_inputs(0), KL | PROB, 0.5, 8, 0),
+        (synth.verify_inputs(2, 40, 20000 + 8 * 37, 29, 0.2, seed=41), KL, 0.5, 4, 1),       # ragged last chunk
+        (synth.verify_inputs(2, 40, 20000 + 8 * 37, 29, 0.2, seed=41), CONF | PROB, 0.5, 4, 2),
+        (synth.verify_inputs(15, 8192, 64, 5700, 0.2, seed=31), KL, 0.5, 40, 3),              # many short rows
+        (synth.verify_inputs(3, 96, 32000, 80, 0.3, seed=42), TRUST, 0.5, 0, 0),
+    ]
+    for (dra, ver, tokens, flags), mode, tau, k, seed in cases:
+        d_in = dra if (mode & 0xFF) == KL else None
+        cta_cap(0)
+        ref = run_gpu(dd, d_in, ver, tokens, flags, mode, tau, k, seed)
+        for cap in (1, 7, 37):
+            cta_cap(cap)
+            got = run_gpu(dd, d_in, ver, tokens, flags, mode, tau, k, seed)
+            for a, b in zip(ref, got):
+                assert np.array_equal(a, b), f"cap {cap}"
+        cta_cap(0)
+        check_verify(*ref, oracle_mod.verify(d_in, ver, tokens, flags, mode, tau, k, seed), flags, tokens)
+
+
+@pytest.mark.parametrize("V", [4096, 20000, 1003])
+def test_excluded_tokens(dd, oracle_mod, V):
+    """Logits of -inf (banned or padded vocabulary entries) at shared and at drafter-only
+    indices: probability zero, no term in Eq. 5; the other rows are untouched by the detour."""
+    ninf = np.uint16(0xFF80)
+    if True:
+        dra, ver, tokens, flags = synth.verify_inputs(2, 12, V, 12, 0.25, seed=51 + V)
+        rng = np.random.default_rng(V)
+        both = rng.choice(V, size=V // 16, replace=False)
+        dra[0, 1, both] = ninf; ver[0, 1, both] = ninf                 # excluded by both models
+        dra[0, 3, both[:50]] = ninf                                    # excluded by the drafter only
+        run_end = 4000 if V > 4096 else 1000
+        dra[1, 5, 8:run_end] = ninf; ver[1, 5, 8:run_end] = ninf       # a whole run of the row
+        dra[1, 7, :V - 3] = ninf; ver[1, 7, :V - 3] = ninf             # nearly everything
+        tokens[:] = np.argmax(synth.bf16_bits_to_f32(dra), axis=2)
+        for mode in (KL, CONF, KL | PROB):
+            _, ref, got = compare(dd, oracle_mod, dra, ver, tokens, flags, mode, 0.5, 3, 7)
+            assert np.isfinite(ref["out_score"]).all() and np.isfinite(got[2]).all()
