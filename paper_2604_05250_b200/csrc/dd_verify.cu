@@ -184,9 +184,9 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
 
 // Counters live in their own allocation: it holds nothing else, so it is all zero whenever no
 // launch is in flight, whatever (B, P) the previous call used.  Its last 256 bytes hold the
-// streaming kernel's three words: health, ticket counter, finished CTAs.
+// streaming kernel's health word.
 constexpr size_t kControlBytes = 256;
-constexpr size_t kStatusOffset = 0, kTicketOffset = 64, kCtasDoneOffset = 128;
+constexpr size_t kStatusOffset = 0;
 
 size_t counter_bytes(int B, int P)
 {
@@ -272,8 +272,7 @@ int launch_stream(const VerifyParams &p, cudaStream_t stream)
         }
     }
     const long units = (long)p.B * p.P * p.nchunks;
-    long grid = (units + kSConsumers - 1) / kSConsumers;
-    if (grid > sms) grid = sms;
+    long grid = units < sms ? units : sms;
     const int cap = g_max_ctas.load(std::memory_order_relaxed);
     if (cap > 0 && grid > cap) grid = cap;
     verify_stream_kernel<KL><<<(unsigned)grid, kSThreads, kSRingBytes, stream>>>(p);
@@ -380,8 +379,6 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     p.seq_counter = (unsigned int *)((char *)ctx->verify_cnt + ((bp * 4 + 255) & ~size_t(255)));
     char *control = (char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes;
     p.status = (unsigned int *)(control + kStatusOffset);
-    p.ticket = (unsigned int *)(control + kTicketOffset);
-    p.ctas_done = (unsigned int *)(control + kCtasDoneOffset);
     char *w = (char *)ctx->verify_ws;
     p.row_score = (float *)w;          w += (bp * 4 + 255) & ~size_t(255);
     p.row_argmax = (int *)w;           w += (bp * 4 + 255) & ~size_t(255);
@@ -493,8 +490,6 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     p.row_counter = (unsigned int *)base;
     p.seq_counter = (unsigned int *)(base + kStaticRowsSlot);
     p.status = (unsigned int *)(control + kStatusOffset);
-    p.ticket = (unsigned int *)(control + kTicketOffset);
-    p.ctas_done = (unsigned int *)(control + kCtasDoneOffset);
     p.row_score = (float *)(base + kStaticCounterBytes);
     p.row_argmax = (int *)(base + kStaticCounterBytes + kStaticRowsSlot);
     p.partials = (Partial *)(base + kStaticCounterBytes + kStaticRowBytes);
@@ -507,7 +502,6 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     // health word is left alone: it is sticky, like dd_verify's).
     DD_CUDA_TRY(cudaMemsetAsync(p.row_counter, 0, bp * 4, s));
     DD_CUDA_TRY(cudaMemsetAsync(p.seq_counter, 0, (size_t)B * 4, s));
-    DD_CUDA_TRY(cudaMemsetAsync(p.ticket, 0, kControlBytes - kTicketOffset, s));
     return launch(p, streaming, s);
 }
 

@@ -47,8 +47,6 @@ struct VerifyParams {
     int *row_argmax;             // [B*P]
     Partial *partials;           // [B*P*nchunks]
     unsigned int *status;        // one word: first expired wait of the streaming kernel (may be null)
-    unsigned int *ticket;        // streaming kernel: units drawn beyond the fixed first ones (zero at rest)
-    unsigned int *ctas_done;     // streaming kernel: CTAs that have drawn their last ticket (zero at rest)
 };
 
 __device__ __forceinline__ float ex2_approx(float x)

@@ -300,16 +300,17 @@ __device__ __noinline__ void fold_partials(const Partial *src, int n, float &sco
     sv = warp_sum(sv);
     if (KL) { sd = warp_sum(sd); tt = warp_sum(tt); }
     float sc = 0.f;
-    if (lane == 0) {
-        if (KL) {
-            const double lse_v = (double)Mv * kLn2 + log(sv);
-            const double lse_d = (double)Md * kLn2 + log(sd);
-            const double kl = tt / sd - lse_d + lse_v;
+    if (KL) {
+        // lane 0 takes the verifier's logarithm while lane 1 takes the drafter's
+        const double lse = (lane == 0 ? (double)Mv : (double)Md) * kLn2 + log(lane == 0 ? sv : sd);
+        const double lse_d = __shfl_sync(0xFFFFFFFFu, lse, 1);
+        if (lane == 0) {
+            const double kl = tt / sd - lse_d + lse;
             sc = (float)fmax(kl, 0.0);
-        } else {
-            // the maximum's own term is 2^(m*log2e - M), not exactly 1
-            sc = (float)(exp2((double)bm_v * (double)kLog2e - (double)Mv) / sv);
         }
+    } else if (lane == 0) {
+        // the maximum's own term is 2^(m*log2e - M), not exactly 1
+        sc = (float)(exp2((double)bm_v * (double)kLog2e - (double)Mv) / sv);
     }
     score = __shfl_sync(0xFFFFFFFFu, sc, 0);
     argmax = bidx;

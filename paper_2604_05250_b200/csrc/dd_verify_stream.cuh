@@ -1,22 +1,23 @@
 // Streaming kernel of dd_verify (V % 8 == 0, 16-byte aligned logits).
 //
-// One persistent CTA per SM: sixteen consumer warps, one producer warp, one publishing warp.
+// One persistent CTA per SM: fifteen streaming warps and one publishing warp.
 //
 // Work.  A flagged row is cut into chunks of a fixed number of logits (a multiple of the stage
-// size); the (row, chunk) units of all flagged rows are numbered in row order.  A unit is the
-// work of one consumer warp and yields one partial.  The first two units of every consumer are
-// fixed by its position in the grid; every further one is drawn from a global ticket counter,
-// one unit ahead of need, so a warp that streams faster simply takes more units.  Which warp
-// computes a unit never changes the unit's partial, and rows are folded from their partials
-// in chunk order, so the results do not depend on the grid or on timing.
+// size); the (row, chunk) units of all flagged rows, numbered in row order, are cut into equal
+// contiguous ranges, one per CTA (more, taken in rounds, when a range would not fit the CTA's
+// table).  A unit is the work of one streaming warp and yields one partial; inside the CTA the
+// range's units go to whichever warp asks next.  Which warp computes a unit never changes the
+// unit's partial, and rows are folded from their partials in chunk order, so the results
+// depend neither on the grid nor on timing.
 //
-// Data path.  Lane w of the producer warp feeds consumer warp w: it maps the consumer's next
-// unit to its row, and for every stage-sized piece of the unit (1024 logits of both tensors,
-// or 2048 of the verifier alone: 4 KB) issues bulk asynchronous copies from global memory into
-// the consumer's private ring of stages in shared memory, completing on the stage's "full"
-// mbarrier.  The consumer waits for the stage, loads its eight 16-byte vectors per lane, hands
-// the stage back (the "empty" mbarrier) as soon as the first pass has consumed the registers,
-// and accumulates.  Consumers do no address arithmetic and no global loads.
+// Data path.  Every streaming warp owns a ring of three 4 KB stages in shared memory.  One lane
+// issues bulk asynchronous copies from global memory into a stage (1024 logits of both
+// tensors, or 2048 of the verifier alone), completing on the stage's mbarrier; the warp waits
+// for the stage, loads its eight 16-byte vectors per lane, and as soon as the first pass has
+// consumed the registers the same lane re-arms the stage with the piece three steps ahead.
+// The copy instructions run on the warp-uniform datapath: issued by one lane they cost a few
+// dozen cycles per piece, issued by a separate warp on behalf of fifteen others they
+// serialised into thousands.  No lane computes a global address in the arithmetic.
 //
 // Arithmetic.  Within a chunk every lane keeps its own state: packed bf16x2 running maxima of
 // the verifier with the ordinal of the word where each half first rose (the lowest index of
@@ -24,31 +25,36 @@
 // T = sum 2^(..)(l_D - l_V) against reference points fixed by the lane's first piece of the
 // chunk (any reference works as long as it is reused; an overflow of the range shows up as a
 // non-finite sum and sends the chunk to a careful scalar path, as do logits of -inf).  Lanes
-// talk to each other only when the chunk ends: the 32 lane states become one partial, which
-// goes to the publishing warp through a queue in shared memory.
+// talk to each other only when the chunk ends: the 32 lane states become one partial in the
+// CTA's table in shared memory.
 //
-// Publication.  The publishing warp stores partials to global memory in batches, counts them
-// per row (one fence per batch), folds the rows it completes in chunk order in fp64 (Eq. 5,
-// Eq. 7), counts rows per sequence and decides the sequences it completes (Section 3.2).
+// Rows.  The warp that stores the last chunk of a row's share of the range folds the row
+// there, in chunk order in fp64 (Eq. 5, Eq. 7): a row that lies inside one range costs no
+// global round trip.  The two rows a range may share with its neighbours go through global
+// memory (their partials, one fence and one counter update per range; the last arriver folds
+// the same partials in the same order), and their units are handed out first, so that they are
+// complete long before the range is.  The publishing warp takes finished rows from a queue in
+// shared memory, stores their scores, counts them per sequence (one fence and one counter
+// update per sequence and range) and decides the sequences it completes (Section 3.2).
 #pragma once
 
 #include "dd_verify_common.cuh"
 
 namespace ddv {
 
-constexpr int kSConsumers = 16;                               // warps that compute
-constexpr int kSProducerWarp = kSConsumers;                   // one warp that issues the copies
-constexpr int kSPublisherWarp = kSConsumers + 1;              // one warp that publishes partials
-constexpr int kSWarps = kSConsumers + 2;
+constexpr int kSConsumers = 15;                               // warps that stream
+constexpr int kSPublisherWarp = kSConsumers;                  // one warp that publishes finished rows
+constexpr int kSWarps = kSConsumers + 1;
 constexpr int kSThreads = kSWarps * 32;
-constexpr int kSStages = 3;                                   // ring slots per consumer
+constexpr int kSStages = 3;                                   // ring slots per streaming warp
 constexpr int kSStageBytes = 4096;
 constexpr int kSRingBytes = kSConsumers * kSStages * kSStageBytes;
-constexpr int kSQueue = 64;                                   // finished-unit queue slots
+constexpr int kSQueue = 64;                                   // finished-row queue slots
+constexpr int kSTable = 640;                                  // chunk partials a CTA keeps per range
 constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per stage (KL)
 constexpr int kMaxPiecesPerChunk = 8;
 constexpr int kSChunk = kPiece * kMaxPiecesPerChunk;          // coarsest cut of a row: 8192 logits
-constexpr unsigned kErrWaitQueue = 0x800, kErrWaitFull = 0x900, kErrWaitEmpty = 0xA00, kErrWaitUnit = 0xB00;
+constexpr unsigned kErrWaitQueue = 0x800, kErrWaitFull = 0x900;
 
 // Logits per tensor in one stage.  Without a drafter tensor (TRUST, CONF) the half of the stage
 // that would hold the drafter's logits holds 1024 more of the verifier's.
@@ -279,47 +285,44 @@ __device__ __noinline__ Partial careful_chunk_partial(const uint16_t *verifier_r
     return c;
 }
 
-// A finished (row, chunk) unit, handed from a consumer warp to the publishing warp.
-struct __align__(16) UnitEvent {
-    int row, chunk, pad0, pad1;
-    Partial part;
+// A finished row (or a range's share of a row cut by a range boundary), handed from a
+// streaming warp to the publishing warp.
+struct __align__(16) RowEvent {
+    int row;
+    int whole;        // 1: the row lay inside the range and is folded: score and argmax are final
+    float score;
+    int argmax;
+    int first_slot;   // whole == 0: the range's chunks of this row are table slots first_slot ..
+    int first_chunk;  //             and chunks first_chunk .. of the row,
+    int count;        //             count of them
+    int pad;
 };
 
-// Queue of unit events between the consumer warps (many producers) and the publishing warp
+// Queue of row events between the streaming warps (many producers) and the publishing warp
 // (one consumer), in shared memory.
 struct EventQueue {
-    UnitEvent entry[kSQueue];
+    RowEvent entry[kSQueue];
     unsigned int ready[kSQueue];     // sequence number + 1 of the entry the slot holds
     unsigned int tail;               // next sequence number to hand out
     unsigned int head;               // entries below this have been taken
-    unsigned int done;               // consumer warps that have finished
-    unsigned int pad;
+    unsigned int done;               // streaming warps that have finished the current range
+    unsigned int next_unit;          // units of the current range handed out so far
 };
 
-// A consumer warp hands over a unit (every lane holds the same partial).  False if the queue
-// stayed full.
-__device__ __forceinline__ bool queue_push(EventQueue &q, int row, int chunk, const Partial &part, int lane)
+// One lane of a streaming warp hands over an entry.  False if the queue stayed full.
+__device__ __forceinline__ bool queue_push(EventQueue &q, const RowEvent &e)
 {
-    int ok = 1;
-    if (lane == 0) {
-        const unsigned int seq = atomicAdd(&q.tail, 1u);
-        volatile unsigned int *head = &q.head;
-        unsigned it = 0;
-        while (seq - *head >= (unsigned)kSQueue) {
-            if (++it > (1u << 22)) { ok = 0; break; }
-            __nanosleep(64);
-        }
-        if (ok) {
-            UnitEvent *e = &q.entry[seq % kSQueue];
-            float4 *dst = reinterpret_cast<float4 *>(e);
-            dst[0] = make_float4(__int_as_float(row), __int_as_float(chunk), 0.f, 0.f);
-            dst[1] = make_float4(part.m_v, part.s_v, __int_as_float(part.idx), part.m_d);
-            dst[2] = make_float4(part.s_d, part.t, 0.f, 0.f);
-            __threadfence_block();
-            *(volatile unsigned int *)&q.ready[seq % kSQueue] = seq + 1u;
-        }
+    const unsigned int seq = atomicAdd(&q.tail, 1u);
+    volatile unsigned int *head = &q.head;
+    unsigned it = 0;
+    while (seq - *head >= (unsigned)kSQueue) {
+        if (++it > (1u << 22)) return false;
+        __nanosleep(64);
     }
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+    q.entry[seq % kSQueue] = e;
+    __threadfence_block();
+    *(volatile unsigned int *)&q.ready[seq % kSQueue] = seq + 1u;
+    return true;
 }
 
 }  // namespace ddv
