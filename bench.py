@@ -9,8 +9,15 @@ followed by one dd_verify call (KL mode), on the LLaDA-8B-shaped workload
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 Prints ONE JSON line (rank 0).  `value` is the device-timed latency of a step
-with the inputs resident in HBM; `e2e` is the same step through the host-buffer
-entry points with the host<->device copies inside the timed region.
+with the inputs resident in HBM: the K steps are captured as one CUDA graph that
+is replayed until the timed window is at least a quarter of a second, every
+replay between two CUDA events, and the median over replays is reported (with
+the 10th and 90th percentiles, and the eagerly launched latency beside it).
+`e2e` is the same step through the host-buffer entry points with the
+host<->device copies inside the timed region.  At one GPU the line also carries
+`other_configs`: every other workload shape (batched serving, long context, the
+sequence-length and vocabulary sweeps, the tiny case, the drafter's block
+attention), each timed the same way with its own clock record.
 --impl reference times the CPU oracle on the host cores instead (a deliberately
 slow baseline, not a target).
 """
@@ -141,6 +148,46 @@ def graph_chunk(K, cap=200):
     return g
 
 
+def percentiles(per_unit_ms):
+    a = np.asarray(per_unit_ms, dtype=np.float64)
+    return {"median": float(np.median(a)), "p10": float(np.percentile(a, 10)), "p90": float(np.percentile(a, 90)),
+            "mean": float(a.mean()), "replays": int(a.size)}
+
+
+def replay_timed(stream, enqueue, units_per_replay, min_window_s=0.25, min_replays=10, max_replays=2000,
+                 barrier=None):
+    """Device time of `enqueue()` (which puts `units_per_replay` units of work on `stream`), repeated
+    until the timed window is at least `min_window_s`; every repetition lies between two CUDA
+    events recorded on `stream`.  Returns (per-unit ms of every repetition, (t0, t1) host window)."""
+    import torch
+    with torch.cuda.stream(stream):
+        enqueue()                                        # untimed: a graph's first replay pays the upload
+        stream.synchronize()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        enqueue()
+        p1.record(stream)
+        stream.synchronize()
+        probe_ms = max(p0.elapsed_time(p1), 1e-3)
+        reps = int(min(max_replays, max(min_replays, math.ceil(1e3 * min_window_s / probe_ms))))
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        if barrier is not None:
+            barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        events[0].record(stream)
+        for r in range(reps):
+            enqueue()
+            events[r + 1].record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        if barrier is not None:
+            barrier()
+        t1 = time.perf_counter()
+    per_unit = [events[r].elapsed_time(events[r + 1]) / units_per_replay for r in range(reps)]
+    return per_unit, (t0, t1)
+
+
 def max_over_ranks(values, device, distributed):
     """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest rank)."""
     import torch
@@ -227,6 +274,181 @@ def run_reference(args):
 # ----------------------------------------------------------------------------- GPU arm
 
 
+def graph_of(stream, fn, n):
+    """Captures fn(0..n-1) on `stream` into a CUDA graph; returns (graph, launches per replay)."""
+    import torch
+    from paper_2604_05250_b200 import binding as dd
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        c0 = dd.launch_count()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(n):
+                fn(i)
+        launches = dd.launch_count() - c0
+    return graph, launches
+
+
+def rotation(bytes_per_set, cap=24):
+    """How many distinct input sets make consecutive launches miss L2."""
+    return max(2, min(cap, int(2.2 * L2_BYTES // max(1, bytes_per_set)) + 1))
+
+
+def device_logits(B, P, V, err, gen, want_drafter):
+    """Logits drawn on the device by the recipe of synth.verify_inputs (verifier N(0, 2^2) with +8 at
+    one token per position; drafter = verifier + N(0, 0.5^2), or an independent N(0, 2^2) row on a
+    share `err` of the positions), rounded to bf16."""
+    import torch
+    dev = gen.device
+    ver = torch.randn(B, P, V, device=dev, generator=gen)
+    ver *= 2.0
+    hot = torch.randint(0, V, (B, P, 1), device=dev, generator=gen)
+    ver.scatter_add_(2, hot, torch.full((B, P, 1), 8.0, device=dev))
+    dra = None
+    if want_drafter:
+        dra = torch.randn(B, P, V, device=dev, generator=gen)
+        wrong = torch.rand(B, P, 1, device=dev, generator=gen) < err
+        dra = torch.where(wrong, 2.0 * dra, ver + 0.5 * dra).to(torch.bfloat16)
+    return dra, ver.to(torch.bfloat16)
+
+
+def other_configs(dd, stream, sampler, peaks, quick=False):
+    """Every workload shape other than the headline step, one entry each: median device time per
+    launch over graph replays, algorithmic TFLOP/s or GB/s, roofline fractions, clocks."""
+    import torch
+    dev = torch.device("cuda", torch.cuda.current_device())
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4242)
+    out = []
+    window = 0.1 if quick else 0.25
+
+    def record(name, op, shape, enqueue_one, n_sets, flops, nbytes, bound, note=None):
+        # a graph of enough launches to last a few milliseconds, replayed over the window
+        with torch.cuda.stream(stream):
+            for i in range(3):
+                enqueue_one(i)
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            enqueue_one(0)
+            e1.record(stream)
+            stream.synchronize()
+        one_ms = max(e0.elapsed_time(e1), 2e-3)
+        n = int(min(200, max(n_sets, math.ceil(4.0 / one_ms))))
+        n = ((n + n_sets - 1) // n_sets) * n_sets if n_sets <= 24 else n
+        graph, launches = graph_of(stream, enqueue_one, n)
+        per_launch, win = replay_timed(stream, graph.replay, n, min_window_s=window)
+        st = percentiles(per_launch)
+        sec = st["median"] * 1e-3
+        entry = {"name": name, "op": op, "shape": shape, "ms": st["median"], "p10": st["p10"], "p90": st["p90"],
+                 "replays": st["replays"], "launches_per_replay": n, "kernels_per_launch": launches // n,
+                 "bound": bound, "clocks": sampler.summary(*win)}
+        if flops:
+            tf = flops / sec / 1e12
+            entry.update(tflops=tf, frac_of_measured_burst=tf / peaks["bf16"],
+                         frac_of_measured_sustained=tf / peaks["bf16_sustained"], frac_of_nominal_2250=tf / NOMINAL_BF16_TFLOPS)
+        if nbytes:
+            gb = nbytes / sec / 1e9
+            entry.update(gbs=gb, algorithmic_bytes=nbytes, frac_of_measured_hbm=gb / peaks["hbm"],
+                         frac_of_nominal_8000=gb / NOMINAL_HBM_GBS)
+        if note:
+            entry["note"] = note
+        out.append(entry)
+        del graph
+
+    # ---- attention: the other configurations and the sequence-length sweep (H = 32, D = 128)
+    att_shapes = [("cfg0 tiny", 1, 4, 128, 64, False), ("cfg2 batched serving", 16, 32, 512, 128, False),
+                  ("cfg3 long context, planted rank-16 structure", 1, 32, 8192, 128, True)]
+    att_shapes += [(f"sweep N={N}", 16384 // N, 32, N, 128, False) for N in synth.ATTENTION_SWEEP_N]
+    att_shapes.append(("B=4 x N=1024", 4, 32, 1024, 128, False))
+    for name, B, H, N, D, planted in att_shapes:
+        per_set = 4 * B * H * N * D * 2
+        ns = rotation(per_set)
+        sets = []
+        for _ in range(ns):
+            q, k, v = (torch.randn(B, H, N, D, device=dev, generator=gen) for _ in range(3))
+            if planted:
+                # a shared rank-16 component of strength 3 in q and k (orthonormal W per head)
+                w = torch.linalg.qr(torch.randn(B, H, D, 16, device=dev, generator=gen))[0].transpose(2, 3)
+                q = q + 3.0 * torch.randn(B, H, N, 16, device=dev, generator=gen) @ w
+                k = k + 3.0 * torch.randn(B, H, N, 16, device=dev, generator=gen) @ w
+            sets.append(tuple(t.to(torch.bfloat16) for t in (q, k, v)))
+        o = torch.empty(B, H, N, D, device=dev, dtype=torch.bfloat16)
+
+        def call(i, sets=sets, o=o, D=D):
+            q, k, v = sets[i % len(sets)]
+            dd.bidir_attention(q, k, v, out=o, scale=D ** -0.5)
+        flops = 4.0 * B * H * N * N * D
+        bound = "tensor" if N >= 1024 else "hbm"
+        record(name, "dd_bidir_attention", dict(B=B, H=H, N=N, D=D), call, ns, flops, float(per_set), bound,
+               note=f"{ns} input sets in rotation" + ("; launch-bound" if N <= 128 else ""))
+        del sets, o
+    assert dd.attention_status() == 0
+
+    # ---- the drafter's shape: a block of queries over stored keys
+    for name, B, Nq, Nkv in [("drafter block B=64", 64, 32, 1024), ("drafter block B=16", 16, 32, 1024),
+                             ("drafter block Nq=128 Nkv=4096", 16, 128, 4096)]:
+        H, D = 32, 128
+        per_set = (2 * Nkv + 2 * Nq) * B * H * D * 2
+        ns = rotation(per_set)
+        sets = [tuple(torch.randn(B, H, n, D, device=dev, generator=gen).to(torch.bfloat16) for n in (Nq, Nkv, Nkv))
+                for _ in range(ns)]
+        o = torch.empty(B, H, Nq, D, device=dev, dtype=torch.bfloat16)
+
+        def call(i, sets=sets, o=o):
+            q, k, v = sets[i % len(sets)]
+            dd.block_attention(q, k, v, out=o)
+        record(name, "dd_block_attention", dict(B=B, H=H, Nq=Nq, Nkv=Nkv, D=D), call, ns,
+               4.0 * B * H * Nq * Nkv * D, float(per_set), "hbm" if Nq <= 256 else "tensor")
+        del sets, o
+    assert dd.attention_status() == 0
+
+    # ---- verification: the other configurations and the vocabulary / masked-count sweep
+    T, K_, C = synth.MODE_TRUST, synth.MODE_KL, synth.MODE_CONF
+    ver_shapes = [("cfg0 tiny", 1, 128, 1024, 32, 0.10, 8, (T, K_, C)),
+                  ("cfg2 batched serving", 16, 256, 126464, "uniform_25_100", 0.10, 16, (C,)),
+                  ("cfg3 long context", 1, 512, 126464, "all", 0.10, 32, (T, K_))]
+    for V in synth.VERIFY_SWEEP["V"]:
+        for nflag in synth.VERIFY_SWEEP["flagged"]:
+            modes = (T, K_, C) if (V == 126464 and nflag == 512) else (K_,)
+            ver_shapes.append((f"sweep V={V} masked={nflag}", 1, 512, V, nflag, 0.20, 8 if nflag == 32 else 32, modes))
+    mode_name = {T: "TRUST", K_: "KL", C: "CONF"}
+    for name, B, P, V, flagged, err, k, modes in ver_shapes:
+        want_d = K_ in modes
+        counts = synth.flag_counts(B, P, flagged, np.random.default_rng(7))
+        flags_h = np.zeros((B, P), dtype=np.uint8)
+        for b in range(B):
+            flags_h[b, np.sort(np.random.default_rng(b).choice(P, size=counts[b], replace=False))] = 1
+        n_flagged = int(flags_h.sum())
+        flags = torch.from_numpy(flags_h).to(dev)
+        per_set = n_flagged * V * 2 * (2 if want_d else 1)
+        ns = rotation(per_set, cap=8)
+        if B * P * V * 2 > (1 << 30):
+            ns = 1                                   # one set is already many times the L2
+        sets = [device_logits(B, P, V, err, gen, want_d) for _ in range(ns)]
+        tokens = torch.randint(0, V, (B, P), device=dev, dtype=torch.int32, generator=gen)
+        ot = torch.empty(B, P, device=dev, dtype=torch.int32)
+        om = torch.empty(B, P, device=dev, dtype=torch.uint8)
+        osc = torch.empty(B, P, device=dev, dtype=torch.float32)
+        for mode in modes:
+            def call(i, sets=sets, mode=mode):
+                dra, ver = sets[i % len(sets)]
+                dd.verify(dra if mode == K_ else None, ver, tokens, flags, mode, 0.5, k, 0,
+                          out_tokens=ot, out_mask=om, out_score=osc)
+            nbytes = n_flagged * V * 2.0 * (2 if mode == K_ else 1) + B * P * 14.0
+            record(f"{name} {mode_name[mode]}", "dd_verify", dict(B=B, P=P, V=V, flagged_rows=n_flagged, mode=mode_name[mode], k=k),
+                   call, max(1, ns), 0.0, nbytes, "hbm",
+                   note=(f"{ns} input sets in rotation" if ns > 1 else "one set, larger than the L2 many times over") +
+                        ("; under 20 us: launch-bound" if nbytes < 2e7 else ""))
+        if name.startswith("cfg2"):
+            def call_u(i, sets=sets):
+                dd.unmask(sets[i % len(sets)][1], tokens, flags, 0.5, 16, out_tokens=ot, out_mask=om, out_conf=osc)
+            record("cfg2 shape, drafter's unmasking step", "dd_unmask", dict(B=B, P=P, V=V, masked_rows=n_flagged, k=16),
+                   call_u, 1, 0.0, n_flagged * V * 2.0 + B * P * 14.0, "hbm")
+        del sets
+    assert dd.verify_status() == 0
+    return out
+
+
 def run_ours(args):
     import torch
     rank, local_rank, world = dist_env()
@@ -238,6 +460,7 @@ def run_ours(args):
     if distributed:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+    barrier = (lambda: dist.barrier()) if distributed else None
 
     from paper_2604_05250_b200 import binding as dd
     from paper_2604_05250_b200 import build
@@ -282,55 +505,39 @@ def run_ours(args):
         verify_call(i)
 
     stream = torch.cuda.Stream(device=dev)
-
-    def timed(fn, n, use_graph=True):
-        """Device time (ms) of n calls fn(0..n-1) on `stream`, CUDA events on that stream."""
-        g = graph_chunk(n)
-        launches = 0
-        with torch.cuda.stream(stream):
-            if use_graph:
-                graph = torch.cuda.CUDAGraph()
-                c0 = dd.launch_count()
-                with torch.cuda.graph(graph, stream=stream):
-                    for i in range(g):
-                        fn(i)
-                launches = (dd.launch_count() - c0) * (n // g)
-                graph.replay()                      # untimed: first replay pays the upload
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            stream.synchronize()
-            if distributed:
-                dist.barrier()
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            e0.record(stream)
-            if use_graph:
-                for _ in range(n // g):
-                    graph.replay()
-            else:
-                c0 = dd.launch_count()
-                for i in range(n):
-                    fn(i)
-                launches = dd.launch_count() - c0
-            e1.record(stream)
-            stream.synchronize()
-            torch.cuda.synchronize()
-            if distributed:
-                dist.barrier()
-            t1 = time.perf_counter()
-        return e0.elapsed_time(e1), launches, (t0, t1)
-
     sampler.start()
     with torch.cuda.stream(stream):
         for i in range(W):
             step(i)
     stream.synchronize()
-    assert dd.attention_status() == 0
+    assert dd.attention_status() == 0 and dd.verify_status() == 0
 
-    use_graph = not args.no_graph
-    total_ms, launches, window = timed(step, K, use_graph)
-    att_ms, _, _ = timed(attention_call, K, use_graph)
-    ver_ms, _, _ = timed(verify_call, K, use_graph)
+    # ---- the K steps as a CUDA graph (in pieces of at most 200 steps), replayed over the window
+    g = graph_chunk(K)
+
+    def graph_runner(fn):
+        graph, launches = graph_of(stream, fn, g)
+
+        def run():
+            for _ in range(K // g):
+                graph.replay()
+        return run, launches * (K // g), graph
+
+    run_step, launches_per_pass, _g1 = graph_runner(step)
+    per_step, window = replay_timed(stream, run_step, K, barrier=barrier)
+    run_att, _, _g2 = graph_runner(attention_call)
+    per_att, _ = replay_timed(stream, run_att, K, barrier=barrier)
+    run_ver, _, _g3 = graph_runner(verify_call)
+    per_ver, _ = replay_timed(stream, run_ver, K, barrier=barrier)
     clocks = sampler.summary(*window)
+
+    # ---- the same steps launched eagerly through the C ABI (tensor maps encoded per call)
+    eager_n = min(K, 200)
+
+    def eager():
+        for i in range(eager_n):
+            step(i)
+    per_eager, _ = replay_timed(stream, eager, eager_n, min_window_s=0.1, barrier=barrier)
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region
     pin = lambda a: torch.from_numpy(a).pin_memory()  # noqa: E731
@@ -362,26 +569,39 @@ def run_ours(args):
         e1.record(stream)
         stream.synchronize()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    sampler.stop()
     h2d = 3 * attention_bytes() / 4 + 2 * VER["B"] * VER["P"] * VER["V"] * 2 + VER["B"] * VER["P"] * 5
     d2h = attention_bytes() / 4 + VER["B"] * VER["P"] * 9
-    assert dd.attention_status() == 0
+    assert dd.attention_status() == 0 and dd.verify_status() == 0
 
-    # ---- max over ranks
-    total_ms, att_ms, ver_ms, e2e_ms = max_over_ranks([total_ms, att_ms, ver_ms, e2e_ms], dev, distributed)
-    ms_step, att_step, ver_step = total_ms / K, att_ms / K, ver_ms / K
+    # ---- max over ranks of every statistic
+    st_step, st_att, st_ver, st_eager = (percentiles(x) for x in (per_step, per_att, per_ver, per_eager))
+    keys = ("median", "p10", "p90", "mean")
+    flat = [st[k] for st in (st_step, st_att, st_ver, st_eager) for k in keys] + [e2e_ms]
+    flat = max_over_ranks(flat, dev, distributed)
+    for n, st in enumerate((st_step, st_att, st_ver, st_eager)):
+        for m, k in enumerate(keys):
+            st[k] = flat[4 * n + m]
+    e2e_ms = flat[-1]
+    ms_step, att_step, ver_step = st_step["median"], st_att["median"], st_ver["median"]
 
     if rank == 0:
         peaks = measured_peaks()
-        long_loop = att_ms > 1000.0
-        att_peak = peaks["bf16_sustained"] if long_loop else peaks["bf16"]
+        others = None
+        if world == 1 and not args.no_other_configs:
+            del att_dev, ver_dev
+            torch.cuda.empty_cache()
+            others = other_configs(dd, stream, sampler, peaks, quick=args.quick)
+        sampler.stop()
+        att_peak = peaks["bf16"]
         att_tflops = attention_flops() / (att_step * 1e-3) / 1e12
         ver_gbs = verify_bytes(n_flagged) / (ver_step * 1e-3) / 1e9
         kernels = {
-            "attention": {"ms": att_step, "tflops": att_tflops, "frac_of_nominal_2250": att_tflops / NOMINAL_BF16_TFLOPS,
+            "attention": {"ms": att_step, "p10": st_att["p10"], "p90": st_att["p90"], "tflops": att_tflops,
+                          "frac_of_nominal_2250": att_tflops / NOMINAL_BF16_TFLOPS,
                           "frac_of_measured": att_tflops / att_peak,
-                          "peak_used": f"{att_peak} TFLOP/s ({'sustained' if long_loop else 'burst'}, {peaks['source']})"},
-            "verify": {"ms": ver_step, "gbs": ver_gbs, "frac_of_nominal_8000": ver_gbs / NOMINAL_HBM_GBS,
+                          "peak_used": f"{att_peak} TFLOP/s (burst, {peaks['source']})"},
+            "verify": {"ms": ver_step, "p10": st_ver["p10"], "p90": st_ver["p90"], "gbs": ver_gbs,
+                       "frac_of_nominal_8000": ver_gbs / NOMINAL_HBM_GBS,
                        "frac_of_measured": ver_gbs / peaks["hbm"], "algorithmic_bytes": verify_bytes(n_flagged),
                        "peak_used": f"{peaks['hbm']} GB/s ({peaks['source']})"},
         }
@@ -401,17 +621,26 @@ def run_ours(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "l2": f"inputs rotate over {att_sets} attention sets and {ver_sets} "
                        "logit sets, each group larger than 2x L2, so every step reads HBM",
-                       "launch": "cuda_graph replay" if use_graph else "eager", "parallelism": f"replicas x{world}"},
+                       "launch": f"cuda_graph of {K} steps, replayed {st_step['replays']} times; value = median over replays",
+                       "parallelism": f"replicas x{world}"},
+            "latency": {"median_ms": st_step["median"], "p10_ms": st_step["p10"], "p90_ms": st_step["p90"],
+                        "mean_ms": st_step["mean"], "replays": st_step["replays"],
+                        "eager_median_ms": st_eager["median"], "eager_p10_ms": st_eager["p10"],
+                        "eager_p90_ms": st_eager["p90"]},
             "throughput": {"value": world * 1e3 / ms_step, "unit": "verify_steps/s"},
             "clocks": clocks,
             "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "steps": e2e_steps},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(launches_per_pass * st_step["replays"]),
             "roofline": roof,
             "kernels": kernels,
             "cpu_baseline": cpu,
         }
+        if others is not None:
+            line["other_configs"] = others
         print(json.dumps(line), flush=True)
+    else:
+        sampler.stop()
     if distributed:
         dist.barrier()
         dist.destroy_process_group()
@@ -421,10 +650,11 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--no-other-configs", action="store_true", help="time the headline step only")
+    ap.add_argument("--quick", action="store_true", help="shorter timing windows for the other configurations")
     args = ap.parse_args()
     if args.steps < 1:
         ap.error("--steps must be >= 1")

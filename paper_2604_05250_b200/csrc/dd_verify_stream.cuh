@@ -10,11 +10,11 @@
 // unit's partial, and rows are folded from their partials in chunk order, so the results
 // depend neither on the grid nor on timing.
 //
-// Data path.  Every streaming warp owns a ring of three 4 KB stages in shared memory.  One lane
+// Data path.  Every streaming warp owns a ring of two 4 KB stages in shared memory.  One lane
 // issues bulk asynchronous copies from global memory into a stage (1024 logits of both
 // tensors, or 2048 of the verifier alone), completing on the stage's mbarrier; the warp waits
 // for the stage, loads its eight 16-byte vectors per lane, and as soon as the first pass has
-// consumed the registers the same lane re-arms the stage with the piece three steps ahead.
+// consumed the registers the same lane re-arms the stage with the piece two steps ahead.
 // The copy instructions run on the warp-uniform datapath: issued by one lane they cost a few
 // dozen cycles per piece, issued by a separate warp on behalf of fifteen others they
 // serialised into thousands.  No lane computes a global address in the arithmetic.
@@ -46,7 +46,7 @@ constexpr int kSConsumers = 15;                               // warps that stre
 constexpr int kSPublisherWarp = kSConsumers;                  // one warp that publishes finished rows
 constexpr int kSWarps = kSConsumers + 1;
 constexpr int kSThreads = kSWarps * 32;
-constexpr int kSStages = 3;                                   // ring slots per streaming warp
+constexpr int kSStages = 2;                                   // ring slots per streaming warp (three gain nothing)
 constexpr int kSStageBytes = 4096;
 constexpr int kSRingBytes = kSConsumers * kSStages * kSStageBytes;
 constexpr int kSQueue = 64;                                   // finished-row queue slots

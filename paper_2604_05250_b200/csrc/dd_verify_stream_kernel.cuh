@@ -19,6 +19,7 @@ __device__ __forceinline__ int count_flagged(const VerifyParams &p, int b)
 struct Pending {
     int b;          // this lane's sequence, -1: none
     int cnt;        // finished rows of that sequence not reported yet
+    int target;     // flagged rows of that sequence (counted when the sequence first shows up)
     int used;       // lanes in use (the same in every lane)
 };
 
@@ -34,13 +35,14 @@ __device__ __forceinline__ void pending_flush(const VerifyParams &p, Pending &pe
     for (int e = 0; e < pend.used; ++e) {
         const int b = __shfl_sync(full, pend.b, e);
         const unsigned after = __shfl_sync(full, before, e) + (unsigned)__shfl_sync(full, pend.cnt, e);
-        if (after != (unsigned)count_flagged(p, b)) continue;
+        if (after != (unsigned)__shfl_sync(full, pend.target, e)) continue;
         __threadfence();
         if ((threadIdx.x & 31) == 0) p.seq_counter[b] = 0u;      // ready for the next launch
         decide_sequence(p, b, stage);
     }
     pend.b = -1;
     pend.cnt = 0;
+    pend.target = 0;
     pend.used = 0;
 }
 
@@ -55,9 +57,11 @@ __device__ __forceinline__ void pending_add(const VerifyParams &p, Pending &pend
         return;
     }
     if (pend.used == 32) pending_flush(p, pend, stage);
+    const int target = count_flagged(p, b);
     if (lane == pend.used) {
         pend.b = b;
         pend.cnt = cnt;
+        pend.target = target;
     }
     ++pend.used;
 }
@@ -123,6 +127,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     Pending pend;
     pend.b = -1;
     pend.cnt = 0;
+    pend.target = 0;
     pend.used = 0;
     bool rehearsed = false;
     // sequences without a single flagged row pass through; this CTA's share of them
@@ -344,7 +349,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                         }
                         break;
                     }
-                    __nanosleep(100);
+                    __nanosleep(32);
                     continue;
                 }
                 idle = 0;

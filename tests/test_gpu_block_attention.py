@@ -149,7 +149,7 @@ def test_argument_errors(dd):
 
 @pytest.mark.parametrize("layout", ["bhnd", "bnhd"])
 def test_drafter_shape_full_size(dd, oracle_mod, layout):
-    """The shape bench_ops times: 32 queries over 1024 stored keys, B = 16, H = 32, D = 128."""
+    """The drafter shape bench.py times: 32 queries over 1024 stored keys, B = 16, H = 32, D = 128."""
     B, H, Nq, Nkv, D = 16, 32, 32, 1024, 128
     q, k, v = block_inputs(B, H, Nq, Nkv, D, 77)
     kv_len = np.random.default_rng(3).integers(Nkv // 4, Nkv + 1, size=B).astype(np.int32)

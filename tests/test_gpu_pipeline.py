@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 
 from paper_2604_05250_b200 import synth
+from tests._toy_models import ToyModel
 from tests._parity import to_torch_bf16
 
 pytestmark = pytest.mark.gpu
@@ -26,8 +27,8 @@ def problem(seed, B=3, P=40, prompt=8):
     target = rng.integers(0, V - 1, size=(B, P)).astype(np.int32)     # MASK_ID never is a target
     start = np.full((B, P), MASK_ID, dtype=np.int32)
     start[:, :prompt] = target[:, :prompt]
-    drafter = synth.ToyModel(target, V, MASK_ID, seed + 1, wrong_share=0.2, base=1.0, gain=4.0)
-    verifier = synth.ToyModel(target, V, MASK_ID, seed + 2, wrong_share=0.0, base=3.0, gain=6.0)
+    drafter = ToyModel(target, V, MASK_ID, seed + 1, wrong_share=0.2, base=1.0, gain=4.0)
+    verifier = ToyModel(target, V, MASK_ID, seed + 2, wrong_share=0.0, base=3.0, gain=6.0)
     return target, start, drafter, verifier
 
 

@@ -2,6 +2,7 @@
 import numpy as np
 
 from paper_2604_05250_b200 import synth
+from tests._toy_models import ToyModel
 
 MASK_ID, V = 63, 64
 
@@ -11,8 +12,8 @@ def problem(seed, B=2, P=30, prompt=6, wrong=0.25):
     target = rng.integers(0, V - 1, size=(B, P)).astype(np.int32)
     start = np.full((B, P), MASK_ID, dtype=np.int32)
     start[:, :prompt] = target[:, :prompt]
-    drafter = synth.ToyModel(target, V, MASK_ID, seed + 1, wrong_share=wrong, base=1.0, gain=4.0)
-    verifier = synth.ToyModel(target, V, MASK_ID, seed + 2, wrong_share=0.0, base=3.0, gain=6.0)
+    drafter = ToyModel(target, V, MASK_ID, seed + 1, wrong_share=wrong, base=1.0, gain=4.0)
+    verifier = ToyModel(target, V, MASK_ID, seed + 2, wrong_share=0.0, base=3.0, gain=6.0)
     return target, start, drafter, verifier
 
 
