@@ -270,6 +270,9 @@ int launch_stream(const VerifyParams &p, cudaStream_t stream)
         if (!g_smem_attr_done[dev][KL ? 1 : 0]) {
             DD_CUDA_TRY(cudaFuncSetAttribute(verify_stream_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSRingBytes));
+            // the same split of the SM's memory as the attention kernel that runs before and after
+            DD_CUDA_TRY(cudaFuncSetAttribute(verify_stream_kernel<KL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             cudaSharedmemCarveoutMaxShared));
             g_smem_attr_done[dev][KL ? 1 : 0] = true;
         }
     }

@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             // ---- lane 0 feeds the ring: the piece it will issue next
             int i_row = 0, i_chunk = 0, i_piece = 0, i_npieces = 0, i_where = 0;
             bool i_more = true;               // false once the end marker has been posted
+            const uint64_t policy = l2_evict_first_policy();
             auto issue = [&](unsigned stage) {
                 if (!i_more) return;
                 const uint32_t bar = s_addr(&s_full[warp][stage]);
@@ -202,8 +203,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 const uint32_t dst = ring + stage * kSStageBytes;
                 const size_t off = (size_t)i_row * p.V + e_begin;
                 sbar_expect_tx(bar, KL ? 2u * bytes : bytes);
-                bulk_load(dst, p.verifier + off, bytes, bar);
-                if (KL) bulk_load(dst + kSStageBytes / 2, p.drafter + off, bytes, bar);
+                bulk_load(dst, p.verifier + off, bytes, bar, policy);
+                if (KL) bulk_load(dst + kSStageBytes / 2, p.drafter + off, bytes, bar, policy);
                 ++i_piece;
             };
             if (lane == 0) {
