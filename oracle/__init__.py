@@ -55,6 +55,11 @@ def _load():
         lib.dd_oracle_verify.argtypes = [vp, vp, vp, vp, i32, f64, i32, u64,
                                          vp, vp, vp, vp, i32, i32, i32]
         lib.dd_oracle_verify.restype = i32
+        lib.dd_oracle_verify_f64.argtypes = [vp, vp, vp, vp, i32, f64, i32, u64,
+                                             vp, vp, vp, vp, i32, i32, i32]
+        lib.dd_oracle_verify_f64.restype = i32
+        lib.dd_oracle_lm_head.argtypes = [vp, vp, vp, i32, i32, i32, vp]
+        lib.dd_oracle_lm_head.restype = None
         lib.dd_oracle_unmask.argtypes = [vp, vp, vp, f64, i32, vp, vp, vp, vp, i32, i32, i32]
         lib.dd_oracle_unmask.restype = None
         lib.dd_oracle_threads.argtypes = []
@@ -185,6 +190,69 @@ def verify(drafter, verifier, tokens, flags, mode, tau, k, seed):
     if rc != 0:
         raise ValueError(f"dd_oracle_verify rejected its arguments (rc={rc})")
     return dict(out_tokens=out_tokens, out_mask=out_mask, out_score=out_score, exempt=exempt)
+
+
+def lm_head(hidden, weight, flags=None):
+    """Logits of the language-model head: hidden [rows,K] x weight [V,K]^T in fp64 (uint16 bf16 bits in).
+    Rows with flag 0 are skipped (zeros).  Returns float64 [rows,V]."""
+    hidden, weight = _u16(hidden), _u16(weight)
+    rows, K = hidden.shape
+    V = weight.shape[0]
+    assert weight.shape == (V, K)
+    if flags is not None:
+        flags = np.ascontiguousarray(flags, dtype=np.uint8).reshape(rows)
+    out = np.empty((rows, V), dtype=np.float64)
+    _load().dd_oracle_lm_head(_ptr(hidden), _ptr(weight), _ptr(flags), rows, K, V, _ptr(out))
+    return out
+
+
+def verify_f64(drafter, verifier, tokens, flags, mode, tau, k, seed):
+    """Verification algorithm A on fp64 logits [B,P,V] (what a fused language-model head hands over
+    without rounding).  Same outputs as verify()."""
+    verifier = np.ascontiguousarray(verifier, dtype=np.float64)
+    B, P, V = verifier.shape
+    if drafter is not None:
+        drafter = np.ascontiguousarray(drafter, dtype=np.float64)
+        assert drafter.shape == verifier.shape
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    flags = np.ascontiguousarray(flags, dtype=np.uint8)
+    assert tokens.shape == (B, P) and flags.shape == (B, P)
+    out_tokens = np.empty((B, P), dtype=np.int32)
+    out_mask = np.empty((B, P), dtype=np.uint8)
+    out_score = np.empty((B, P), dtype=np.float64)
+    exempt = np.empty((B, P), dtype=np.uint8)
+    rc = _load().dd_oracle_verify_f64(_ptr(drafter), _ptr(verifier), _ptr(tokens), _ptr(flags),
+                                      int(mode), float(np.float32(tau)), int(k), int(seed),
+                                      _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), _ptr(exempt), B, P, V)
+    if rc != 0:
+        raise ValueError(f"dd_oracle_verify_f64 rejected its arguments (rc={rc})")
+    return dict(out_tokens=out_tokens, out_mask=out_mask, out_score=out_score, exempt=exempt)
+
+
+def lm_head_verify(hidden_d, weight_d, hidden_v, weight_v, tokens, flags, mode, tau, k, seed, round_logits=False):
+    """The verification phase from the models' last hidden states: logits by lm_head(), then the
+    verification algorithm.  hidden_* [B,P,K], weight_* [V,K] (uint16 bf16 bits; the drafter pair may
+    be None unless the mode is KL).  round_logits: round the logits to bf16 first (what an unfused
+    head stores) and run verify() on them; otherwise verify_f64() on the fp64 logits.
+    Adds `top2_gap` [B,P]: difference of the two largest verifier logits (token ids are only
+    comparable where it exceeds what fp32 accumulation can blur)."""
+    B, P, K = hidden_v.shape
+    fl = np.ascontiguousarray(flags, dtype=np.uint8)
+    lv = lm_head(np.ascontiguousarray(hidden_v).reshape(B * P, K), weight_v, fl)
+    ld = None
+    if hidden_d is not None:
+        ld = lm_head(np.ascontiguousarray(hidden_d).reshape(B * P, K), weight_d, fl)
+    V = lv.shape[1]
+    part = np.partition(lv, V - 2, axis=1)
+    gap = (part[:, V - 1] - part[:, V - 2]).reshape(B, P)
+    if round_logits:
+        to_bits = lambda a: ((a.astype(np.float32).view(np.uint32) + (((a.astype(np.float32).view(np.uint32) >> 16) & 1) + 0x7FFF)) >> 16).astype(np.uint16)
+        r = verify(None if ld is None else to_bits(ld).reshape(B, P, V), to_bits(lv).reshape(B, P, V),
+                   tokens, flags, mode, tau, k, seed)
+    else:
+        r = verify_f64(None if ld is None else ld.reshape(B, P, V), lv.reshape(B, P, V), tokens, flags, mode, tau, k, seed)
+    r["top2_gap"] = gap
+    return r
 
 
 def unmask(logits, tokens, flags, tau, k):

@@ -33,6 +33,10 @@
  *                              that the paper does not fix: PARITY UNPINNED
  *                              for those two (checked only against a brute
  *                              force restatement of the same reading).
+ *   dd_oracle_lm_head          pinned   (identity and one-hot weights, numpy fp64
+ *                                        matmul); dd_oracle_verify_f64 is
+ *                                        dd_oracle_verify's algorithm on fp64 logits
+ *                                        (pinned against it on bf16-exact logits)
  *   dd_oracle_unmask           pinned for the threshold rule and the fixed
  *                              number per step (hand-built cases, scipy
  *                              softmax + numpy argsort on random inputs,
@@ -239,18 +243,18 @@ double dd_oracle_uniform(uint64_t seed, int b, int i)
  *   kl       : KL(p_D || p_V) = sum_x p_D(x) (ln p_D(x) - ln p_V(x)) (Eq. 5),
  *              natural log, clamped at zero; 0 if drafter row is NULL.
  */
-void dd_oracle_row_scores(const uint16_t *drafter_row, const uint16_t *verifier_row,
-                          int V, int32_t *argmax_v, double *conf, double *kl)
+static void row_scores_f64(const double *drafter_row, const double *verifier_row,
+                           int V, int32_t *argmax_v, double *conf, double *kl)
 {
     /* verifier: argmax and log-softmax */
     int a = 0;
-    double mv = bf16_to_f64(verifier_row[0]);
+    double mv = verifier_row[0];
     for (int x = 1; x < V; ++x) {
-        const double l = bf16_to_f64(verifier_row[x]);
+        const double l = verifier_row[x];
         if (l > mv) { mv = l; a = x; }
     }
     double zv = 0.0;
-    for (int x = 0; x < V; ++x) zv += exp(bf16_to_f64(verifier_row[x]) - mv);
+    for (int x = 0; x < V; ++x) zv += exp(verifier_row[x] - mv);
     const double lse_v = mv + log(zv);
     *argmax_v = a;
     *conf = exp(mv - lse_v);
@@ -259,15 +263,15 @@ void dd_oracle_row_scores(const uint16_t *drafter_row, const uint16_t *verifier_
     if (drafter_row) {
         double md = -INFINITY;
         for (int x = 0; x < V; ++x) {
-            const double l = bf16_to_f64(drafter_row[x]);
+            const double l = drafter_row[x];
             if (l > md) md = l;
         }
         double zd = 0.0;
-        for (int x = 0; x < V; ++x) zd += exp(bf16_to_f64(drafter_row[x]) - md);
+        for (int x = 0; x < V; ++x) zd += exp(drafter_row[x] - md);
         const double lse_d = md + log(zd);
         for (int x = 0; x < V; ++x) {
-            const double log_pd = bf16_to_f64(drafter_row[x]) - lse_d;
-            const double log_pv = bf16_to_f64(verifier_row[x]) - lse_v;
+            const double log_pd = drafter_row[x] - lse_d;
+            const double log_pv = verifier_row[x] - lse_v;
             /* a token the drafter excludes (logit -inf, p_D(x) = 0) adds nothing: the
              * Kullback-Leibler sum of Eq. 5 runs over the support of p_D (0 ln 0 = 0) */
             if (log_pd == -INFINITY) continue;
@@ -276,6 +280,21 @@ void dd_oracle_row_scores(const uint16_t *drafter_row, const uint16_t *verifier_
         if (acc < 0.0) acc = 0.0;
     }
     *kl = acc;
+}
+
+/* The same for rows stored as bf16: converted exactly, then the arithmetic above. */
+void dd_oracle_row_scores(const uint16_t *drafter_row, const uint16_t *verifier_row,
+                          int V, int32_t *argmax_v, double *conf, double *kl)
+{
+    double *v = (double *)malloc(sizeof(double) * (size_t)V);
+    double *d = drafter_row ? (double *)malloc(sizeof(double) * (size_t)V) : NULL;
+    for (int x = 0; x < V; ++x) {
+        v[x] = bf16_to_f64(verifier_row[x]);
+        if (d) d[x] = bf16_to_f64(drafter_row[x]);
+    }
+    row_scores_f64(d, v, V, argmax_v, conf, kl);
+    free(v);
+    free(d);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -297,17 +316,18 @@ enum { FLAG_PROBABILISTIC = 0x100, FLAG_EMIT_DRAFTER = 0x200 };
  *
  * Returns 0, or -1 on an unknown mode.
  */
-int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
-                     const int32_t *tokens, const uint8_t *flags,
-                     int mode, double tau, int k, uint64_t seed,
-                     int32_t *out_tokens, uint8_t *out_mask, double *out_score,
-                     uint8_t *exempt, int B, int P, int V)
+static int verify_core(const uint16_t *drafter, const uint16_t *verifier,
+                       const double *drafter_f64, const double *verifier_f64,
+                       const int32_t *tokens, const uint8_t *flags,
+                       int mode, double tau, int k, uint64_t seed,
+                       int32_t *out_tokens, uint8_t *out_mask, double *out_score,
+                       uint8_t *exempt, int B, int P, int V)
 {
     const int algo = mode & 0xFF;
     const int probabilistic = (mode & FLAG_PROBABILISTIC) != 0;
     const int emit_drafter = (mode & FLAG_EMIT_DRAFTER) != 0;
     if (algo != MODE_TRUST && algo != MODE_KL && algo != MODE_CONF) return -1;
-    if (algo == MODE_KL && !drafter) return -1;
+    if (algo == MODE_KL && !drafter && !drafter_f64) return -1;
 
     const long BP = (long)B * P;
     int32_t *amax = (int32_t *)malloc(sizeof(int32_t) * (size_t)BP);
@@ -319,9 +339,14 @@ int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
     for (long t = 0; t < BP; ++t) {
         amax[t] = 0; conf[t] = 0.0; kl[t] = 0.0;
         if (!flags[t]) continue;
-        const uint16_t *dv = verifier + (size_t)t * V;
-        const uint16_t *dd = (algo == MODE_KL) ? drafter + (size_t)t * V : NULL;
-        dd_oracle_row_scores(dd, dv, V, &amax[t], &conf[t], &kl[t]);
+        if (verifier_f64) {      /* logits handed over in fp64 (the fused language-model head) */
+            const double *dd = (algo == MODE_KL) ? drafter_f64 + (size_t)t * V : NULL;
+            row_scores_f64(dd, verifier_f64 + (size_t)t * V, V, &amax[t], &conf[t], &kl[t]);
+        } else {
+            const uint16_t *dv = verifier + (size_t)t * V;
+            const uint16_t *dd = (algo == MODE_KL) ? drafter + (size_t)t * V : NULL;
+            dd_oracle_row_scores(dd, dv, V, &amax[t], &conf[t], &kl[t]);
+        }
     }
 
     int *members = (int *)malloc(sizeof(int) * (size_t)P);
@@ -416,6 +441,50 @@ int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
     free(members); free(rel); free(rank);
     free(amax); free(conf); free(kl);
     return 0;
+}
+
+int dd_oracle_verify(const uint16_t *drafter, const uint16_t *verifier,
+                     const int32_t *tokens, const uint8_t *flags,
+                     int mode, double tau, int k, uint64_t seed,
+                     int32_t *out_tokens, uint8_t *out_mask, double *out_score,
+                     uint8_t *exempt, int B, int P, int V)
+{
+    return verify_core(drafter, verifier, NULL, NULL, tokens, flags, mode, tau, k, seed,
+                       out_tokens, out_mask, out_score, exempt, B, P, V);
+}
+
+/* The same algorithm on logits given in fp64, [B,P,V] (drafter may be NULL unless the mode is KL). */
+int dd_oracle_verify_f64(const double *drafter, const double *verifier,
+                         const int32_t *tokens, const uint8_t *flags,
+                         int mode, double tau, int k, uint64_t seed,
+                         int32_t *out_tokens, uint8_t *out_mask, double *out_score,
+                         uint8_t *exempt, int B, int P, int V)
+{
+    if (!verifier) return -1;
+    return verify_core(NULL, NULL, drafter, verifier, tokens, flags, mode, tau, k, seed,
+                       out_tokens, out_mask, out_score, exempt, B, P, V);
+}
+
+/* ------------------------------------------------------------------------ */
+/* The language-model head of the verification phase: Algorithm 1 computes p_V(. | x^D) "for all
+ * positions", i.e. logits[t, x] = sum_k hidden[t, k] * weight[x, k] (the last hidden state of
+ * position t against the output embedding of token x), softmax over x.  hidden [rows, K] and weight
+ * [V, K] are bf16 bit patterns; the sum is taken in fp64, in index order.  Rows whose flag is 0 are
+ * skipped (left at 0) when flags is not NULL.                                                      */
+void dd_oracle_lm_head(const uint16_t *hidden, const uint16_t *weight, const uint8_t *flags,
+                       int rows, int K, int V, double *logits)
+{
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int t = 0; t < rows; ++t) {
+        for (int x = 0; x < V; ++x) {
+            double acc = 0.0;
+            if (!flags || flags[t]) {
+                const uint16_t *h = hidden + (size_t)t * K, *w = weight + (size_t)x * K;
+                for (int j = 0; j < K; ++j) acc += bf16_to_f64(h[j]) * bf16_to_f64(w[j]);
+            }
+            logits[(size_t)t * V + x] = acc;
+        }
+    }
 }
 
 /* ------------------------------------------------------------------------ */
