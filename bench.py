@@ -50,7 +50,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (None until a capture of that kernel exists).
-NCU_TRAFFIC_BYTES = {"attention": 25.27e6, "verify": 136.55e6}
+NCU_TRAFFIC_BYTES = {"attention": 25.27e6, "verify": 134.7e6}
 
 
 def attention_flops():
@@ -449,6 +449,48 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
     return out
 
 
+def run_eager_other(dd, which, K, W):
+    """K eagerly launched calls of one entry point on one of the other shapes (for profilers)."""
+    import torch
+    dev = torch.device("cuda", torch.cuda.current_device())
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    if which == "drafter_block":
+        B, H, Nq, Nkv, D = 64, 32, 32, 1024, 128
+        sets = [tuple(torch.randn(B, H, n, D, device=dev, generator=gen).to(torch.bfloat16) for n in (Nq, Nkv, Nkv))
+                for _ in range(2)]
+        o = torch.empty(B, H, Nq, D, device=dev, dtype=torch.bfloat16)
+        name = f"dd_block_attention B={B} H={H} Nq={Nq} Nkv={Nkv} D={D}"
+
+        def call(i):
+            q, k, v = sets[i % 2]
+            dd.block_attention(q, k, v, out=o)
+    else:
+        B, P, V = VER["B"], VER["P"], VER["V"]
+        sets = [device_logits(B, P, V, 0.1, gen, False)[1] for _ in range(5)]
+        tokens = torch.zeros(B, P, device=dev, dtype=torch.int32)
+        flags = torch.ones(B, P, device=dev, dtype=torch.uint8)
+        ot, om = torch.empty_like(tokens), torch.empty_like(flags)
+        oc = torch.empty(B, P, device=dev, dtype=torch.float32)
+        name = f"dd_unmask on logits [{B},{P},{V}], every position masked"
+
+        def call(i):
+            dd.unmask(sets[i % 5], tokens, flags, 0.5, 8, out_tokens=ot, out_mask=om, out_conf=oc)
+    for i in range(W):
+        call(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        call(i)
+    e1.record()
+    torch.cuda.synchronize()
+    assert dd.attention_status() == 0 and dd.verify_status() == 0
+    print(json.dumps({"mode": "eager-only", "workload": name, "steps": K, "warmup": W,
+                      "ms_per_call": e0.elapsed_time(e1) / K}), flush=True)
+    return 0
+
+
 def run_ours(args):
     import torch
     rank, local_rank, world = dist_env()
@@ -468,6 +510,8 @@ def run_ours(args):
     dd.lib()
 
     K, W = args.steps, max(3, args.warmup)
+    if args.eager_only in ("drafter_block", "unmask_cfg1"):
+        return run_eager_other(dd, args.eager_only, K, W)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
 
     # ---- inputs: several distinct sets per kernel so that consecutive steps never hit L2
@@ -511,6 +555,26 @@ def run_ours(args):
             step(i)
     stream.synchronize()
     assert dd.attention_status() == 0 and dd.verify_status() == 0
+
+    if args.eager_only:
+        # K eagerly launched steps and nothing else: the command profilers are pointed at
+        with torch.cuda.stream(stream):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0 = dd.launch_count()
+            e0.record(stream)
+            for i in range(K):
+                step(i)
+            e1.record(stream)
+            stream.synchronize()
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"mode": "eager-only", "workload": WORKLOAD, "steps": K, "warmup": W,
+                              "ms_per_step": e0.elapsed_time(e1) / K, "gpu_launches": int(dd.launch_count() - c0)}),
+                  flush=True)
+        if distributed:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
 
     # ---- the K steps as a CUDA graph (in pieces of at most 200 steps), replayed over the window
     g = graph_chunk(K)
@@ -655,6 +719,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-other-configs", action="store_true", help="time the headline step only")
     ap.add_argument("--quick", action="store_true", help="shorter timing windows for the other configurations")
+    ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1"],
+                    help="launch K steps (or calls on one of two other shapes) eagerly and exit: for profilers")
     args = ap.parse_args()
     if args.steps < 1:
         ap.error("--steps must be >= 1")

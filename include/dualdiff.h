@@ -45,7 +45,7 @@ typedef enum {
     DD_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, unknown mode, NaN tau, k < 0 */
     DD_ERR_UNSUPPORTED = -2, /* valid request outside what the kernels implement          */
     DD_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed; see dd_last_cuda_error  */
-    DD_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see dd_attention_status) */
+    DD_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see dd_clear_status)    */
 } dd_status;
 
 /* `mode` argument of dd_verify: algorithm in the low 8 bits, flag bits above. */
@@ -210,20 +210,28 @@ int dd_debug_set_max_ctas(int max_ctas);
 size_t dd_verify_workspace_bytes(int B, int P, int V);
 
 /*
- * Device-side health word of the attention kernel for the current device: 0 if
- * no bounded wait has ever expired, otherwise a non-zero code identifying the
- * wait that gave up (the affected output tile is then undefined).  Synchronises
- * the device.  Returns DD_OK / DD_ERR_TIMEOUT / DD_ERR_CUDA.
+ * Health of the kernels.  Every device-side wait is bounded; a wait that expires records a code in
+ * a per-device health word (one for the attention kernel, one for dd_verify / dd_unmask /
+ * dd_verify_static) and the affected outputs of that launch are undefined.  The word is sticky:
+ *   - the code is also written to a host copy, so the NEXT call of an entry point of that kernel
+ *     on the device returns DD_ERR_TIMEOUT without launching anything and without synchronising
+ *     (dd_verify_static consults the host copy only if another entry point has created it);
+ *   - dd_attention_status() / dd_verify_status() synchronise the device and read the word itself:
+ *     DD_OK, DD_ERR_TIMEOUT (dd_last_cuda_error() names the code) or DD_ERR_CUDA;
+ *   - dd_clear_status() synchronises the device and re-arms both words (the scratch stays
+ *     allocated); dd_release() frees everything.
  */
 int dd_attention_status(void);
+int dd_verify_status(void);
+int dd_clear_status(void);
 
 /*
- * Device-side health word of dd_verify for the current device, with the same
- * meaning and return values as dd_attention_status: non-zero once a bounded wait
- * for a shared-memory copy or queue has expired (the outputs of that call are
- * undefined; dd_release() returns the scratch to its initial state).
+ * Test hook for the above: launches, on `stream`, a one-thread kernel that waits on a barrier
+ * nothing completes, gives up after a few hundred polls (microseconds) and records the expiry in
+ * the health word of the attention kernel (which = 0) or of dd_verify (which = 1) exactly as those
+ * kernels would.  It stalls nothing and faults nothing.  DD_ERR_INVALID_ARG for another `which`.
  */
-int dd_verify_status(void);
+int dd_debug_expire_wait(int which, void *stream);
 
 /* Number of kernels launched by this library in this process (all devices). */
 uint64_t dd_launch_count(void);

@@ -23,7 +23,7 @@ DD_LAYOUT_BHND, DD_LAYOUT_BNHD = 0, 1
 EXPORTS = (
     "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_unmask", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
-    "dd_status_string", "dd_last_cuda_error", "dd_version", "dd_debug_set_max_ctas",
+    "dd_status_string", "dd_last_cuda_error", "dd_version", "dd_debug_set_max_ctas", "dd_clear_status", "dd_debug_expire_wait",
 )
 
 
@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.dd_verify_workspace_bytes.restype = ctypes.c_size_t
         L.dd_launch_count.argtypes = []
         L.dd_launch_count.restype = u64
+        L.dd_clear_status.argtypes = []
+        L.dd_clear_status.restype = i32
+        L.dd_debug_expire_wait.argtypes = [i32, vp]
+        L.dd_debug_expire_wait.restype = i32
         L.dd_debug_set_max_ctas.argtypes = [i32]
         L.dd_debug_set_max_ctas.restype = i32
         L.dd_status_string.argtypes = [i32]
@@ -233,6 +237,16 @@ def launch_count() -> int:
 def debug_set_max_ctas(n: int):
     """Test hook: cap the grid of the streaming verify kernel (0 = no cap)."""
     _check(lib().dd_debug_set_max_ctas(int(n)))
+
+
+def clear_status():
+    """Re-arms the kernels' health words on the current device after a recorded timeout."""
+    _check(lib().dd_clear_status())
+
+
+def debug_expire_wait(which: int, stream=None):
+    """Test hook: records an expired wait for the attention kernel (0) or dd_verify (1)."""
+    _check(lib().dd_debug_expire_wait(int(which), _stream_ptr(stream)))
 
 
 def release():

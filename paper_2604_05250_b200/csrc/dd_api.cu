@@ -46,6 +46,29 @@ DeviceCtx *current_ctx(int *device_out)
     return &g_ctx[dev];
 }
 
+int ensure_mirror(DeviceCtx *ctx)
+{
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (ctx->mirror) return DD_OK;
+    void *host = nullptr, *dev = nullptr;
+    DD_CUDA_TRY(cudaHostAlloc(&host, 64, cudaHostAllocMapped));
+    memset(host, 0, 64);
+    DD_CUDA_TRY(cudaHostGetDevicePointer(&dev, host, 0));
+    ctx->mirror_dev = static_cast<unsigned int *>(dev);
+    ctx->mirror = static_cast<volatile unsigned int *>(host);
+    return DD_OK;
+}
+
+int check_mirror(const DeviceCtx *ctx, int which)
+{
+    if (!ctx->mirror) return DD_OK;
+    const unsigned int word = ctx->mirror[which];
+    if (word == 0) return DD_OK;
+    snprintf(g_err, sizeof g_err, "%s kernel: a bounded wait expired earlier on this device (code 0x%08x); "
+             "dd_clear_status() re-arms it", which == 0 ? "attention" : "verify", word);
+    return DD_ERR_TIMEOUT;
+}
+
 int ensure_bytes(void **ptr, size_t *have, size_t need)
 {
     if (need <= *have && *ptr) return DD_OK;
@@ -96,6 +119,7 @@ int dd_release(void)
     if (ctx->verify_cnt) DD_CUDA_TRY(cudaFree(ctx->verify_cnt));
     if (ctx->staging) DD_CUDA_TRY(cudaFree(ctx->staging));
     if (ctx->attn_status) DD_CUDA_TRY(cudaFree(ctx->attn_status));
+    if (ctx->mirror) DD_CUDA_TRY(cudaFreeHost(const_cast<unsigned int *>(ctx->mirror)));
     *ctx = DeviceCtx();
     return DD_OK;
 }

@@ -24,6 +24,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <mutex>
+
 #include "dd_common.cuh"
 #include "dd_ptx.cuh"
 
@@ -50,7 +52,8 @@ struct AttnParams {
     const int *kv_len;         // [B] keys of each sequence that exist (clamped to 0..Nkv), or null: Nkv
     int head_major;            // 1: [B,H,N,D], tensor maps are 3-D over (D, N, B*H); 0: [B,N,H,D], 4-D maps (D, N, H, B)
     float scale_log2;          // scale * log2(e)
-    unsigned int *status;
+    unsigned int *status;      // health word of the attention kernel on this device
+    unsigned int *mirror;      // its copy in mapped host memory (written only when a wait expires)
 };
 
 template <int D>
@@ -65,9 +68,13 @@ struct Smem {
     static constexpr int kTotal = kTmemSlot + 16;
 };
 
-__device__ __forceinline__ void report(unsigned int *status, unsigned code)
+__device__ __forceinline__ void report(const AttnParams &p, unsigned code)
 {
-    atomicCAS(status, 0u, code | (unsigned)(blockIdx.x & 0xFF));
+    const unsigned word = code | (unsigned)(blockIdx.x & 0xFF);
+    if (atomicCAS(p.status, 0u, word) == 0u && p.mirror) {
+        *reinterpret_cast<volatile unsigned int *>(p.mirror) = word;      // the host sees it without a synchronisation
+        __threadfence_system();
+    }
 }
 
 // One key tile of the online softmax for one query row; s[] holds the raw scores.
@@ -302,7 +309,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     l_run = l_run * scale_own + other.y * scale_other;
                 }
             }
-            if (err != 0) report(p.status, err);
+            if (err != 0) report(p, err);
             const bool stores = !(kBlock && split && g == 1);
             if (stores && err == 0) {
                 // ---- epilogue: O / l -> bf16 -> this tile's Q buffer (every MMA that read it has
@@ -377,7 +384,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int item = 0; item < 2 * nkv; ++item) {
                 if (item == 1 && groups > 1) load_q(1);
                 const int slot = item % kStages, use = item / kStages;
-                if (use > 0 && !mbar_wait(bar_kv_empty(slot), (use - 1) & 1)) { report(p.status, kErrWaitSlot); break; }
+                if (use > 0 && !mbar_wait(bar_kv_empty(slot), (use - 1) & 1)) { report(p, kErrWaitSlot); break; }
                 const uint32_t dst = sRing + slot * kTileBytes;
                 const CUtensorMap *tm = (item & 1) ? &tm_v : &tm_k;
                 mbar_expect_tx(bar_kv_full(slot), kTileBytes);
@@ -478,7 +485,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     if (more) mma_commit(bar_kv_empty(item_k % kStages));
                 }
             } while (false);
-            if (err) report(p.status, err);
+            if (err) report(p, err);
         }
     }
 
@@ -546,12 +553,16 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
            const AttnParams &p, cudaStream_t s)
 {
     static bool attr_done[64] = {};
+    static std::mutex attr_mu;
     int dev = 0;
     DD_CUDA_TRY(cudaGetDevice(&dev));
     const int smem = Smem<D>::kTotal + 1024;
-    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        DD_CUDA_TRY(cudaFuncSetAttribute(attention_kernel<D, kBlock>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_done[dev] = true;
+    {
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+            DD_CUDA_TRY(cudaFuncSetAttribute(attention_kernel<D, kBlock>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attr_done[dev] = true;
+        }
     }
     const long grid = (long)p.BH * p.m_blocks;
     attention_kernel<D, kBlock><<<(unsigned)grid, kThreads, smem, s>>>(tq, tk, tv, to, p);
@@ -576,13 +587,15 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
 
     dd::DeviceCtx *ctx = dd::current_ctx();
     if (!ctx) return DD_ERR_CUDA;
+    int rc = dd::ensure_mirror(ctx);
+    if (rc != DD_OK) return rc;
+    if ((rc = dd::check_mirror(ctx, 0)) != DD_OK) return rc;      // an earlier launch gave up a wait: nothing is launched
     if (!ctx->attn_status) {
         DD_CUDA_TRY(cudaMalloc(&ctx->attn_status, 256));
         DD_CUDA_TRY(cudaMemset(ctx->attn_status, 0, 256));
     }
     const bool head_major = layout == DD_LAYOUT_BHND;
     CUtensorMap tq, tk, tv, to;
-    int rc;
     if ((rc = make_tmap(&tq, q, B, H, Nq, D, head_major)) != DD_OK) return rc;
     if ((rc = make_tmap(&tk, k, B, H, Nkv, D, head_major)) != DD_OK) return rc;
     if ((rc = make_tmap(&tv, v, B, H, Nkv, D, head_major)) != DD_OK) return rc;
@@ -595,6 +608,7 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     p.head_major = head_major ? 1 : 0;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->attn_status;
+    p.mirror = ctx->mirror_dev;
     cudaStream_t s = (cudaStream_t)stream;
     const bool general = kv_len != nullptr || !head_major || Nq != Nkv;
     if (general) return D == 64 ? launch<64, true>(tq, tk, tv, to, p, s) : launch<128, true>(tq, tk, tv, to, p, s);

@@ -19,11 +19,23 @@ struct DeviceCtx {
     void *staging = nullptr;        // device copies of host buffers (the *_host calls)
     size_t staging_bytes = 0;
     unsigned int *attn_status = nullptr;  // one word: first expired wait of the attention kernel
+    // Host copy of the two health words (pinned, mapped): [0] attention, [1] verify.  A kernel that
+    // records an expired wait writes the code here as well, so the next call sees it without a
+    // device synchronisation.
+    volatile unsigned int *mirror = nullptr;
+    unsigned int *mirror_dev = nullptr;   // the same two words as the kernels address them
 };
 
 // Returns the context of the current device (creating it on first use), or
 // nullptr after recording a CUDA error.
 DeviceCtx *current_ctx(int *device_out = nullptr);
+
+// Allocates the host copy of the health words on first use (pinned host memory, no device memory).
+int ensure_mirror(DeviceCtx *ctx);
+
+// DD_ERR_TIMEOUT (with error text) if the host copy shows that kernel `which` (0 attention,
+// 1 verify) has recorded an expired wait on this device; DD_OK otherwise.
+int check_mirror(const DeviceCtx *ctx, int which);
 
 // Grows (never shrinks) a scratch buffer; new memory is zero-filled.
 int ensure_bytes(void **ptr, size_t *have, size_t need);

@@ -374,6 +374,8 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
 
     dd::DeviceCtx *ctx = dd::current_ctx();
     if (!ctx) return DD_ERR_CUDA;
+    if ((rc = dd::ensure_mirror(ctx)) != DD_OK) return rc;
+    if ((rc = dd::check_mirror(ctx, 1)) != DD_OK) return rc;      // an earlier launch gave up a wait: nothing is launched
     rc = dd::ensure_bytes(&ctx->verify_ws, &ctx->verify_ws_bytes, workspace_bytes(B, P, p.nchunks));
     if (rc != DD_OK) return rc;
     rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(B, P) + kControlBytes);
@@ -384,6 +386,7 @@ extern "C" int dd_verify(const void *drafter_logits, const void *verifier_logits
     p.seq_counter = (unsigned int *)((char *)ctx->verify_cnt + ((bp * 4 + 255) & ~size_t(255)));
     char *control = (char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes;
     p.status = (unsigned int *)(control + kStatusOffset);
+    p.mirror = ctx->mirror_dev + 1;
     char *w = (char *)ctx->verify_ws;
     p.row_score = (float *)w;          w += (bp * 4 + 255) & ~size_t(255);
     p.row_argmax = (int *)w;           w += (bp * 4 + 255) & ~size_t(255);
@@ -495,6 +498,14 @@ extern "C" int dd_verify_static(const void *drafter_logits, const void *verifier
     p.row_counter = (unsigned int *)base;
     p.seq_counter = (unsigned int *)(base + kStaticRowsSlot);
     p.status = (unsigned int *)(control + kStatusOffset);
+    {
+        // the host copy of the health word is used if an earlier call of another entry point made
+        // it; this entry point allocates nothing, not even pinned host memory
+        dd::DeviceCtx *ctx = dd::current_ctx();
+        if (!ctx) return DD_ERR_CUDA;
+        if ((rc = dd::check_mirror(ctx, 1)) != DD_OK) return rc;
+        p.mirror = ctx->mirror_dev ? ctx->mirror_dev + 1 : nullptr;
+    }
     p.row_score = (float *)(base + kStaticCounterBytes);
     p.row_argmax = (int *)(base + kStaticCounterBytes + kStaticRowsSlot);
     p.partials = (Partial *)(base + kStaticCounterBytes + kStaticRowBytes);
@@ -531,5 +542,68 @@ extern "C" int dd_verify_status(void)
         dd::set_error_text(text);
         return DD_ERR_TIMEOUT;
     }
+    return DD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Recovery and its test hook.
+
+namespace {
+
+// One thread waits on an mbarrier that nothing will ever complete, gives up after a few hundred
+// polls and records the expiry exactly as the real kernels do.  The launch ends by itself within
+// microseconds: this is how the error path is exercised without stalling a GPU.
+__global__ void expire_wait_kernel(unsigned int *status, unsigned int *mirror, unsigned code)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = ddv::s_addr(&bar);
+    ddv::sbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bool arrived = false;
+    for (int spin = 0; spin < 512 && !arrived; ++spin) arrived = ddv::sbar_try_wait(b, 0);
+    if (!arrived && atomicCAS(status, 0u, code) == 0u && mirror) {
+        *reinterpret_cast<volatile unsigned int *>(mirror) = code;
+        __threadfence_system();
+    }
+}
+
+}  // namespace
+
+extern "C" int dd_debug_expire_wait(int which, void *stream)
+{
+    if (which != 0 && which != 1) return DD_ERR_INVALID_ARG;
+    dd::DeviceCtx *ctx = dd::current_ctx();
+    if (!ctx) return DD_ERR_CUDA;
+    int rc = dd::ensure_mirror(ctx);
+    if (rc != DD_OK) return rc;
+    unsigned int *word = nullptr;
+    if (which == 0) {
+        if (!ctx->attn_status) {
+            DD_CUDA_TRY(cudaMalloc(&ctx->attn_status, 256));
+            DD_CUDA_TRY(cudaMemset(ctx->attn_status, 0, 256));
+        }
+        word = ctx->attn_status;
+    } else {
+        rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(1, 1) + kControlBytes);
+        if (rc != DD_OK) return rc;
+        word = (unsigned int *)((char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes + kStatusOffset);
+    }
+    expire_wait_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(word, ctx->mirror_dev + which, 0xE000u + (unsigned)which);
+    DD_CUDA_TRY(cudaGetLastError());
+    return DD_OK;
+}
+
+extern "C" int dd_clear_status(void)
+{
+    dd::DeviceCtx *ctx = dd::current_ctx();
+    if (!ctx) return DD_ERR_CUDA;
+    DD_CUDA_TRY(cudaDeviceSynchronize());
+    if (ctx->attn_status) DD_CUDA_TRY(cudaMemset(ctx->attn_status, 0, sizeof(unsigned int)));
+    if (ctx->verify_cnt)
+        DD_CUDA_TRY(cudaMemset((char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes + kStatusOffset, 0,
+                               sizeof(unsigned int)));
+    if (unsigned char *fixed = static_scratch_if_resolved())
+        DD_CUDA_TRY(cudaMemset(fixed + 2 * kStaticRowsSlot + kStatusOffset, 0, sizeof(unsigned int)));
+    if (ctx->mirror) ctx->mirror[0] = ctx->mirror[1] = 0u;
     return DD_OK;
 }

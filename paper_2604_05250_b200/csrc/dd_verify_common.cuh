@@ -47,7 +47,19 @@ struct VerifyParams {
     int *row_argmax;             // [B*P]
     Partial *partials;           // [B*P*nchunks]
     unsigned int *status;        // one word: first expired wait of the streaming kernel (may be null)
+    unsigned int *mirror;        // its copy in mapped host memory, written only when a wait expires (may be null)
 };
+
+// Records the first expired wait of a launch: in the device word and, so that the host sees it
+// without a synchronisation, in its host copy.
+__device__ __forceinline__ void report_expired(const VerifyParams &p, unsigned code)
+{
+    const unsigned word = code | (unsigned)(blockIdx.x & 0xFF);
+    if (p.status && atomicCAS(p.status, 0u, word) == 0u && p.mirror) {
+        *reinterpret_cast<volatile unsigned int *>(p.mirror) = word;
+        __threadfence_system();
+    }
+}
 
 __device__ __forceinline__ float ex2_approx(float x)
 {

@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             if (lane == 0) {
                 if (err) {
                     *abort_flag = 1;
-                    if (p.status) atomicCAS(p.status, 0u, err | (blockIdx.x & 0xFF));
+                    report_expired(p, err);
                 }
                 __threadfence_block();
                 atomicAdd(&s_queue.done, 1u);
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                     if (++idle > (1u << 23)) {     // the streaming warps never finished
                         if (lane == 0) {
                             *abort_flag = 1;
-                            if (p.status) atomicCAS(p.status, 0u, kErrWaitQueue | (blockIdx.x & 0xFF));
+                            report_expired(p, kErrWaitQueue);
                         }
                         break;
                     }
