@@ -23,7 +23,7 @@ DD_LAYOUT_BHND, DD_LAYOUT_BNHD = 0, 1
 EXPORTS = (
     "dd_bidir_attention", "dd_block_attention", "dd_verify", "dd_unmask", "dd_bidir_attention_host", "dd_verify_host", "dd_verify_static",
     "dd_verify_workspace_bytes", "dd_attention_status", "dd_verify_status", "dd_launch_count", "dd_release",
-    "dd_status_string", "dd_last_cuda_error", "dd_version", "dd_debug_set_max_ctas", "dd_clear_status", "dd_debug_expire_wait",
+    "dd_status_string", "dd_last_cuda_error", "dd_version", "dd_debug_set_max_ctas", "dd_clear_status", "dd_debug_expire_wait", "dd_lm_head_verify",
 )
 
 
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.dd_verify_workspace_bytes.restype = ctypes.c_size_t
         L.dd_launch_count.argtypes = []
         L.dd_launch_count.restype = u64
+        L.dd_lm_head_verify.argtypes = [vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.dd_lm_head_verify.restype = i32
         L.dd_clear_status.argtypes = []
         L.dd_clear_status.restype = i32
         L.dd_debug_expire_wait.argtypes = [i32, vp]
@@ -195,6 +197,35 @@ def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, se
     _check(fn(_ptr(drafter_logits), _ptr(verifier_logits), _ptr(tokens), _ptr(mask_flags),
               int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
               _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, V, _stream_ptr(stream)))
+    return out_tokens, out_mask, out_score
+
+
+def lm_head_verify(verifier_hidden, verifier_weight, tokens, mask_flags, mode, tau, k, seed,
+                   out_tokens=None, out_mask=None, out_score=None, stream=None):
+    """dd_lm_head_verify: the verifier's language-model head fused with the verification algorithm.
+
+    verifier_hidden [B,P,K], verifier_weight [V,K]: torch.bfloat16 device tensors.
+    Returns (out_tokens int32 [B,P], out_mask uint8 [B,P], out_score float32 [B,P])."""
+    import torch
+    B, P, K = verifier_hidden.shape
+    V = verifier_weight.shape[0]
+    _require(verifier_hidden, torch.bfloat16, (B, P, K), True, "verifier_hidden")
+    _require(verifier_weight, torch.bfloat16, (V, K), True, "verifier_weight")
+    _require(tokens, torch.int32, (B, P), True, "tokens")
+    _require(mask_flags, torch.uint8, (B, P), True, "mask_flags")
+    kw = dict(device=verifier_hidden.device)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, P), dtype=torch.int32, **kw)
+    if out_mask is None:
+        out_mask = torch.empty((B, P), dtype=torch.uint8, **kw)
+    if out_score is None:
+        out_score = torch.empty((B, P), dtype=torch.float32, **kw)
+    _require(out_tokens, torch.int32, (B, P), True, "out_tokens")
+    _require(out_mask, torch.uint8, (B, P), True, "out_mask")
+    _require(out_score, torch.float32, (B, P), True, "out_score")
+    _check(lib().dd_lm_head_verify(_ptr(verifier_hidden), _ptr(verifier_weight), _ptr(tokens), _ptr(mask_flags),
+                                   int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                   _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, K, V, _stream_ptr(stream)))
     return out_tokens, out_mask, out_score
 
 

@@ -1,0 +1,263 @@
+// Language-model head fused with the verification algorithm (Algorithm 1, verification phase:
+// the verifier's distribution p_V(. | x^D) "for all positions" goes straight into A(p_D, p_V, x^D)).
+//
+// logits[t, x] = sum_k hidden[t, k] * weight[x, k] is a [rows, K] x [K, V] product whose result,
+// 253 KB per position at the LLaDA vocabulary, is only ever reduced: per row its maximum, the
+// lowest index of the maximum and the softmax normaliser (Eq. 7).  The kernel therefore keeps the
+// product in tensor memory and never stores a logit: a persistent CTA takes work items of
+// 256 rows x N vocabulary entries (N <= 256), accumulates them with tcgen05 MMAs (two
+// accumulators of 128 rows, fp32) from operand tiles that a TMA producer streams through a
+// three-stage ring, and its epilogue warps turn every accumulator row into one partial
+// (maximum, first index, sum 2^(l*log2e - M)) of the same form as the streaming kernel's chunk
+// partials.  Partials go through the same global table, row counters, fp64 row fold and decision
+// stage as dd_verify's, with "chunk" = vocabulary tile.
+//
+//   warps 0-3   epilogue of accumulator 0 (thread = row = tensor-memory lane)
+//   warps 4-7   epilogue of accumulator 1
+//   warp  8     one thread feeds the ring: per 64-wide k-step the two 128-row tiles of the hidden
+//               states and the N-row tile of the weights (2-D tensor maps, 128-byte swizzle, rows
+//               past the end read as zero; no multicast)
+//   warp  9     one thread issues the MMAs and commits them to the ring's and the accumulators'
+//               barriers
+// Included by dd_verify.cu.
+#pragma once
+
+#include <cuda.h>
+
+#include "dd_ptx.cuh"
+#include "dd_verify_common.cuh"
+
+namespace ddlm {
+
+using namespace ddptx;
+
+constexpr int kThreads = 320;
+constexpr int kEpilogueWarps = 8;
+constexpr int kLoadWarp = 8, kMmaWarp = 9;
+constexpr int kRowsPerItem = 256;          // two accumulators of 128 rows
+constexpr int kBlockK = 64;                // one 128-byte swizzled box per k-step
+constexpr int kStages = 3;
+constexpr int kMaxN = 256;
+constexpr uint32_t kTmemCols = 512;        // accumulator 0 in columns [0, N), accumulator 1 in [256, 256 + N)
+constexpr int kATileBytes = 128 * kBlockK * 2;                        // 16 KB: 128 rows x 64 bf16
+constexpr int kStageBytes = 2 * kATileBytes + kMaxN * kBlockK * 2;    // 64 KB
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr unsigned kErrLmFull = 0xC00, kErrLmEmpty = 0xD00, kErrLmAcc = 0xE00;
+
+struct LmParams {
+    int rows, K, V;            // rows = B * P
+    int N;                     // vocabulary entries per work item (a multiple of 32, <= 256)
+    int n_tiles;               // ceil(V / N): the "chunks" of a row
+    int row_blocks;            // ceil(rows / 256)
+};
+
+// Up to 32 rows' partials of one vocabulary tile (lane l holds row `row` and its partial; `kind`:
+// 1 = a flagged row's partial, 0 = an unflagged row, reported to its sequence once, -1 = nothing).
+// One fence for the batch, one count per row; rows whose last tile this was are folded (fp64, tile
+// order) and reported; the warp that completes a sequence decides it.
+__device__ __forceinline__ void publish_rows(const ddv::VerifyParams &p, const ddv::Partial &c, int row, int tile, int kind)
+{
+    const unsigned full = 0xFFFFFFFFu;
+    if (kind == 1) {
+        ddv::Partial *dst = p.partials + (size_t)row * p.nchunks + tile;
+        __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), 0.f));
+        __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+    __threadfence();
+    bool last = false;
+    if (kind == 1) last = atomicAdd(p.row_counter + row, 1u) == (unsigned)(p.nchunks - 1);
+    unsigned todo = __ballot_sync(full, last);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        ddv::fold_row<false>(p, __shfl_sync(full, row, src), nullptr);
+    }
+    todo = __ballot_sync(full, kind == 0);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        ddv::row_done(p, __shfl_sync(full, row, src) / p.P, nullptr);
+    }
+}
+
+// Epilogue warps: every accumulator row becomes one partial.  Columns are visited in index order
+// with a strict comparison, so the index kept is the lowest index of the maximum.
+__device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyParams &p, uint32_t tmem,
+                                         uint32_t bar_acc_full, uint32_t bar_acc_empty,
+                                         volatile uint32_t *abort_flag, int n_items)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int acc = warp >> 2;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;          // this warp's 32 tensor-memory lanes
+    const uint32_t tacc = tmem + lane_off + (uint32_t)acc * 256u;
+    uint32_t n_done = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_done) {
+        const int tile = item / q.row_blocks, rb = item - tile * q.row_blocks;
+        const int row = rb * kRowsPerItem + acc * 128 + (warp & 3) * 32 + lane, col0 = tile * q.N;
+        bool arrived = false;
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (mbar_try_wait(bar_acc_full, n_done & 1)) { arrived = true; break; }
+            if (it > 64) {
+                __nanosleep(64);
+                if (*abort_flag) break;
+            }
+        }
+        if (!arrived) {
+            if (lane == 0) {
+                *abort_flag = 1u;
+                ddv::report_expired(p, kErrLmAcc);
+            }
+            return;
+        }
+        tc_fence_after();
+        float m = -INFINITY, M = -INFINITY, s = 0.f;
+        int idx = 0x7FFFFFFF;
+        for (int cb = 0; cb < q.N / 32; ++cb) {
+            uint32_t r[32];
+            tmem_ld32(tacc + cb * 32, r);
+            tmem_wait_ld();
+            const int valid = q.V - (col0 + cb * 32);                 // columns of this group that exist
+            if (valid <= 0) break;
+            float cm = -INFINITY;
+            int ci = 0;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float v = __uint_as_float(r[i]);
+                if (i < valid && v > cm) { cm = v; ci = i; }
+            }
+            if (cm > m) {
+                const float M_new = cm * ddv::kLog2e;
+                s *= ddv::rescale_factor(M, M_new);
+                m = cm; M = M_new;
+                idx = col0 + cb * 32 + ci;
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < valid) s += ddv::ex2_approx(fmaf(__uint_as_float(r[i]), ddv::kLog2e, -M));
+        }
+        // both accumulators may be overwritten once every epilogue warp has read its lanes
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_empty);
+
+        ddv::Partial c;
+        c.m_v = m; c.s_v = s; c.idx = idx;
+        c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f; c.pad0 = c.pad1 = 0.f;
+        int kind = -1;
+        if (row < q.rows) kind = p.flags[row] ? 1 : (tile == 0 ? 0 : -1);
+        publish_rows(p, c, min(row, q.rows - 1), tile, kind);
+    }
+}
+
+template <int kDummy>
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w,
+               const LmParams q, const ddv::VerifyParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem_dyn[];
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;     // swizzled tiles: 1024-byte aligned
+    unsigned char *smem_gen = smem_dyn + (smem_base - smem_u32(smem_dyn));
+    const uint32_t bars = smem_base + kStages * kStageBytes;
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
+    const uint32_t bar_acc_full = bars + 8u * (2 * kStages), bar_acc_empty = bars + 8u * (2 * kStages + 1);
+    const uint32_t tmem_slot = bars + 8u * (2 * kStages + 2);
+    volatile uint32_t *tmem_slot_gen = reinterpret_cast<volatile uint32_t *>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 2));
+    volatile uint32_t *abort_flag = tmem_slot_gen + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_items = q.n_tiles * q.row_blocks;
+    const int k_steps = q.K / kBlockK;
+
+    if (tid == 0) {
+        prefetch_tmap(&tm_h); prefetch_tmap(&tm_w);
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, kEpilogueWarps);
+        fence_mbar_init();
+        *abort_flag = 0u;
+    }
+    if (warp == 0) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+
+    // a wait that gives up: the code goes to the health word, every role winds down
+    auto give_up = [&](unsigned code) {
+        *abort_flag = 1u;
+        ddv::report_expired(p, code);
+    };
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if (it > 64) {
+                __nanosleep(32);
+                if (*abort_flag) return false;
+            }
+        }
+        return false;
+    };
+
+    if (warp == kLoadWarp && lane == 0) {
+        // ===================================================================== TMA producer
+        uint32_t step = 0;                                    // k-steps issued over all items
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            const int tile = item / q.row_blocks, rb = item - tile * q.row_blocks;
+            const int row0 = rb * kRowsPerItem, col0 = tile * q.N;
+            bool ok = true;
+            for (int ks = 0; ks < k_steps; ++ks, ++step) {
+                const int s = step % kStages;
+                const uint32_t use = step / kStages;
+                if (use > 0 && !wait(bar_empty(s), (use - 1) & 1)) { give_up(kErrLmEmpty); ok = false; break; }
+                const uint32_t dst = smem_base + s * kStageBytes;
+                mbar_expect_tx(bar_full(s), (uint32_t)(2 * kATileBytes + q.N * kBlockK * 2));
+                tma_load_2d(dst, &tm_h, bar_full(s), ks * kBlockK, row0);
+                tma_load_2d(dst + kATileBytes, &tm_h, bar_full(s), ks * kBlockK, row0 + 128);
+                tma_load_2d(dst + 2 * kATileBytes, &tm_w, bar_full(s), ks * kBlockK, col0);
+            }
+            if (!ok) break;
+        }
+    } else if (warp == kMmaWarp && lane == 0) {
+        // ===================================================================== MMA issuer
+        const uint32_t idesc = idesc_bf16(128, q.N, false);
+        uint32_t step = 0, n_done = 0;                        // k-steps consumed, items finished
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_done) {
+            // the epilogue of the previous item has read both accumulators
+            if (n_done > 0 && !wait(bar_acc_empty, (n_done - 1) & 1)) { give_up(kErrLmAcc); break; }
+            tc_fence_after();
+            bool ok = true;
+            for (int ks = 0; ks < k_steps; ++ks, ++step) {
+                const int s = step % kStages;
+                if (!wait(bar_full(s), (step / kStages) & 1)) { give_up(kErrLmFull); ok = false; break; }
+                tc_fence_after();
+                const uint32_t base = smem_base + s * kStageBytes;
+                const uint64_t a0 = smem_desc_sw128(base, 16, 1024), a1 = smem_desc_sw128(base + kATileBytes, 16, 1024);
+                const uint64_t b = smem_desc_sw128(base + 2 * kATileBytes, 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                    const uint32_t off = (uint32_t)(kk * 32) >> 4;            // 16 bf16 = 32 bytes per MMA
+                    mma_ss(tmem, a0 + off, b + off, idesc, (ks > 0 || kk > 0));
+                    mma_ss(tmem + 256, a1 + off, b + off, idesc, (ks > 0 || kk > 0));
+                }
+                mma_commit(bar_empty(s));                                      // the stage is free once these have run
+            }
+            if (!ok) break;
+            mma_commit(bar_acc_full);
+        }
+    } else if (warp < kEpilogueWarps) {
+        epilogue(q, p, tmem, bar_acc_full, bar_acc_empty, abort_flag, n_items);
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait expired: give copies that may still be in flight time to land before the shared
+        // memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    if (warp == 0) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
+}
+
+}  // namespace ddlm

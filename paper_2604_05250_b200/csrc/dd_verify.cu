@@ -31,6 +31,7 @@
 #include <mutex>
 
 #include "dd_verify_stream.cuh"
+#include "dd_lm_head_kernel.cuh"
 
 namespace {
 
@@ -412,6 +413,129 @@ extern "C" int dd_debug_set_max_ctas(int max_ctas)
 {
     if (max_ctas < 0) return DD_ERR_INVALID_ARG;
     g_max_ctas.store(max_ctas, std::memory_order_relaxed);
+    return DD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// dd_lm_head_verify: the verifier's language-model head fused with the verification algorithm.
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// bf16 matrix [n_rows, K], K innermost, as a 2-D tensor map with boxes of 64 columns x box_rows rows,
+// 128-byte swizzle; rows past the end read as zero.
+int make_matrix_tmap(CUtensorMap *m, const void *base, long n_rows, int K, int box_rows)
+{
+    static EncodeTiledFn fn = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!fn) {
+            void *sym = nullptr;
+            cudaDriverEntryPointQueryResult qr;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr) == cudaSuccess &&
+                qr == cudaDriverEntryPointSuccess)
+                fn = reinterpret_cast<EncodeTiledFn>(sym);
+        }
+    }
+    if (!fn) return dd::cuda_fail(cudaErrorSymbolNotFound, "cuTensorMapEncodeTiled entry point");
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)n_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return dd::cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return DD_OK;
+}
+
+// Vocabulary entries per work item: the multiple of 32 (at most 256) for which the slowest CTA
+// of `ctas` has least to do.
+int pick_tile_n(int V, long row_blocks, int ctas)
+{
+    int best = 256;
+    long best_cost = -1;
+    for (int n = 256; n >= 128; n -= 32) {
+        const long items = ((V + n - 1) / n) * row_blocks;
+        const long cost = ((items + ctas - 1) / ctas) * n;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+    }
+    return best;
+}
+
+}  // namespace
+
+extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifier_weight,
+                                 const int32_t *tokens, const uint8_t *mask_flags,
+                                 int mode, float tau, int k, uint64_t seed,
+                                 int32_t *out_tokens, uint8_t *out_mask, float *out_score,
+                                 int B, int P, int K, int V, void *stream)
+{
+    if (!verifier_hidden || !verifier_weight) return DD_ERR_INVALID_ARG;
+    if (K <= 0) return DD_ERR_INVALID_ARG;
+    int rc = check_args(nullptr, verifier_hidden, tokens, mask_flags, mode, tau, k, out_tokens, out_mask, B, P, V);
+    if (rc == DD_ERR_INVALID_ARG && (mode & 0xFF) == DD_MODE_KL) return DD_ERR_UNSUPPORTED;      // the drafter's head is not fused yet
+    if (rc != DD_OK) return rc;
+    if (K % ddlm::kBlockK != 0) return DD_ERR_UNSUPPORTED;
+    if ((((uintptr_t)verifier_hidden | (uintptr_t)verifier_weight) & 15) != 0) return DD_ERR_UNSUPPORTED;
+    const long rows = (long)B * P;
+    const int sms = sm_count_of_current_device();
+    if (sms < 0) return sms;
+    int cap = g_max_ctas.load(std::memory_order_relaxed);
+    const int ctas = cap > 0 && cap < sms ? cap : sms;
+
+    ddlm::LmParams q;
+    q.rows = (int)rows; q.K = K; q.V = V;
+    q.row_blocks = (int)((rows + ddlm::kRowsPerItem - 1) / ddlm::kRowsPerItem);
+    q.N = pick_tile_n(V, q.row_blocks, sms);
+    q.n_tiles = (V + q.N - 1) / q.N;
+    if (rows * q.n_tiles >= (1L << 31) - (1L << 24)) return DD_ERR_UNSUPPORTED;
+
+    VerifyParams p;
+    p.nchunks = q.n_tiles;
+    p.chunk = q.N;
+    dd::DeviceCtx *ctx = dd::current_ctx();
+    if (!ctx) return DD_ERR_CUDA;
+    if ((rc = dd::ensure_mirror(ctx)) != DD_OK) return rc;
+    if ((rc = dd::check_mirror(ctx, 1)) != DD_OK) return rc;
+    rc = dd::ensure_bytes(&ctx->verify_ws, &ctx->verify_ws_bytes, workspace_bytes(B, P, p.nchunks));
+    if (rc != DD_OK) return rc;
+    rc = dd::ensure_bytes(&ctx->verify_cnt, &ctx->verify_cnt_bytes, counter_bytes(B, P) + kControlBytes);
+    if (rc != DD_OK) return rc;
+    const size_t bp = (size_t)rows;
+    p.row_counter = (unsigned int *)ctx->verify_cnt;
+    p.seq_counter = (unsigned int *)((char *)ctx->verify_cnt + ((bp * 4 + 255) & ~size_t(255)));
+    p.status = (unsigned int *)((char *)ctx->verify_cnt + ctx->verify_cnt_bytes - kControlBytes + kStatusOffset);
+    p.mirror = ctx->mirror_dev + 1;
+    char *w = (char *)ctx->verify_ws;
+    p.row_score = (float *)w;          w += (bp * 4 + 255) & ~size_t(255);
+    p.row_argmax = (int *)w;           w += (bp * 4 + 255) & ~size_t(255);
+    p.partials = (Partial *)w;
+    fill_params(p, nullptr, nullptr, tokens, mask_flags, mode, tau, k, seed, out_tokens, out_mask, out_score, B, P, V);
+
+    CUtensorMap tm_h, tm_w;
+    if ((rc = make_matrix_tmap(&tm_h, verifier_hidden, rows, K, 128)) != DD_OK) return rc;
+    if ((rc = make_matrix_tmap(&tm_w, verifier_weight, V, K, q.N)) != DD_OK) return rc;
+
+    int dev = 0;
+    DD_CUDA_TRY(cudaGetDevice(&dev));
+    {
+        static bool attr_done[64] = {};
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!attr_done[dev]) {
+            DD_CUDA_TRY(cudaFuncSetAttribute(ddlm::lm_head_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             ddlm::kSmemBytes));
+            attr_done[dev] = true;
+        }
+    }
+    const long items = (long)q.n_tiles * q.row_blocks;
+    const unsigned grid = (unsigned)(items < ctas ? items : ctas);
+    ddlm::lm_head_kernel<0><<<grid, ddlm::kThreads, ddlm::kSmemBytes, (cudaStream_t)stream>>>(tm_h, tm_w, q, p);
+    DD_CUDA_TRY(cudaGetLastError());
+    dd::count_launch();
     return DD_OK;
 }
 

@@ -47,7 +47,7 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
     const long base = (long)b * p.P;
     const bool kl_mode = p.algo == DD_MODE_KL;
     const int nk = (p.P + 31) / 32;                 // positions per lane (upper bound)
-    const bool staged = p.P <= kDecideKeys;
+    const bool staged = stage != nullptr && p.P <= kDecideKeys;      // without a staging area: re-read from memory
 
     // key of position i: order-preserving image of its reliability, 0 outside the set.
     // Both loads are unconditional (the score slot exists for every position), so a pass

@@ -147,3 +147,28 @@ def attention_config_inputs(config_index: int):
     c = ATTENTION_CONFIGS[config_index]
     return attention_inputs(c["B"], c["H"], c["N"], c["D"], config_seed(config_index),
                             planted=c["planted"])
+
+
+# ----------------------------------------------------------------------------
+# language-model head inputs
+
+
+def lm_head_inputs(B, P, K, V, flagged, seed, bump=8.0):
+    """Last hidden states [B,P,K] and output embedding [V,K] (uint16 bf16 bits) whose product has the
+    statistics of verify_inputs' verifier logits: entries ~ N(0, 2^2), plus about `bump` at one random
+    token per position (the hidden state leans towards that token's embedding).  Stands in for
+    LLaDA-8B's final hidden states and tied output embedding (K = 4096, V = 126464).
+
+    Returns (hidden u16 [B,P,K], weight u16 [V,K], tokens i32 [B,P], flags u8 [B,P])."""
+    rng = np.random.default_rng([int(seed), 0x1E4D])
+    counts = flag_counts(B, P, flagged, rng)
+    weight = rng.standard_normal((V, K), dtype=np.float32)
+    weight *= np.float32(2.0 / np.sqrt(K))
+    hidden = rng.standard_normal((B, P, K), dtype=np.float32)
+    hot = rng.integers(0, V, size=(B, P))
+    hidden += np.float32(bump / 4.0) * weight[hot]               # |w|^2 ~ 4: logit of the hot token rises by ~bump
+    tokens = rng.integers(0, V, size=(B, P)).astype(np.int32)
+    flags = np.zeros((B, P), dtype=np.uint8)
+    for b in range(B):
+        flags[b, np.sort(rng.choice(P, size=counts[b], replace=False))] = 1
+    return f32_to_bf16_bits(hidden), f32_to_bf16_bits(weight), tokens, flags
