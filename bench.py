@@ -446,6 +446,24 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
                    call_u, 1, 0.0, n_flagged * V * 2.0 + B * P * 14.0, "hbm")
         del sets
     assert dd.verify_status() == 0
+
+    # ---- the verifier's language-model head fused with the verification algorithm (K = 4096)
+    for name, B, P in [("fused LM head, cfg1 rows", 1, 256), ("fused LM head, cfg2 rows", 16, 256)]:
+        K, V = 4096, 126464
+        hs = [torch.randn(B, P, K, device=dev, generator=gen).to(torch.bfloat16) for _ in range(2)]
+        ws = [(torch.randn(V, K, device=dev, generator=gen) * (2.0 / K ** 0.5)).to(torch.bfloat16) for _ in range(2)]
+        tokens = torch.zeros(B, P, device=dev, dtype=torch.int32)
+        flags = torch.ones(B, P, device=dev, dtype=torch.uint8)
+        ot, om = torch.empty_like(tokens), torch.empty_like(flags)
+        osc = torch.empty(B, P, device=dev, dtype=torch.float32)
+
+        def call_lm(i, hs=hs, ws=ws):
+            dd.lm_head_verify(hs[i % 2], ws[i % 2], tokens, flags, C, 0.5, 32, 0, out_tokens=ot, out_mask=om, out_score=osc)
+        record(name, "dd_lm_head_verify", dict(B=B, P=P, K=K, V=V, mode="CONF", k=32), call_lm, 2,
+               2.0 * B * P * K * V, float(V * K * 2 + B * P * K * 2), "tensor",
+               note="two weight matrices in rotation (2 x 1.04 GB); bytes = weights and hidden states once")
+        del hs, ws
+    assert dd.verify_status() == 0
     return out
 
 
