@@ -88,6 +88,30 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     // ---- every thread counts the flagged rows of its contiguous slice of the B*P rows; the block
     // scan gives each thread the number of flagged rows before its slice, and the total
     const long n_rows = (long)p.B * p.P;
+    if (warp == kSPublisherWarp && lane < kSConsumers) {
+        // Before anything is known about the flags: ask the L2 (and with it the address translation)
+        // for the first lines this CTA would stream if every row were flagged, one unit per
+        // streaming warp.  The first copies of a launch otherwise arrive up to 4 us apart, and a
+        // CTA that starts late finishes late.  A prefetch has no effect on any result; where the
+        // guess is wrong it is wasted.
+        const unsigned units = (unsigned)n_rows * (unsigned)nch, per = (units + gridDim.x - 1) / gridDim.x;
+        if (per <= (unsigned)kSTable) {
+            const unsigned lo = blockIdx.x * (units / gridDim.x) + min(blockIdx.x, units % gridDim.x);
+            const unsigned hi = lo + units / gridDim.x + (blockIdx.x < units % gridDim.x ? 1u : 0u);
+            if (hi > lo) {
+                const unsigned f_hi = (hi - 1) / (unsigned)nch;
+                unsigned t = (unsigned)lane;
+                if (f_hi > lo / (unsigned)nch && hi < (f_hi + 1) * (unsigned)nch) t += f_hi * (unsigned)nch - lo;
+                if (t >= hi - lo) t -= hi - lo;
+                if (t < hi - lo) {
+                    const unsigned g = lo + t, f = g / (unsigned)nch;
+                    const size_t off = (size_t)f * p.V + (size_t)(g - f * (unsigned)nch) * p.chunk;
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.verifier + off));
+                    if (KL) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.drafter + off));
+                }
+            }
+        }
+    }
     const long slice = (n_rows + kSThreads - 1) / kSThreads;
     const long my_begin = min(n_rows, (long)tid * slice), my_end = min(n_rows, my_begin + slice);
     int my_count = 0;
