@@ -458,10 +458,17 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
         osc = torch.empty(B, P, device=dev, dtype=torch.float32)
 
         def call_lm(i, hs=hs, ws=ws):
-            dd.lm_head_verify(hs[i % 2], ws[i % 2], tokens, flags, C, 0.5, 32, 0, out_tokens=ot, out_mask=om, out_score=osc)
+            dd.lm_head_verify(None, None, hs[i % 2], ws[i % 2], tokens, flags, C, 0.5, 32, 0, out_tokens=ot, out_mask=om, out_score=osc)
         record(name, "dd_lm_head_verify", dict(B=B, P=P, K=K, V=V, mode="CONF", k=32), call_lm, 2,
                2.0 * B * P * K * V, float(V * K * 2 + B * P * K * 2), "tensor",
                note="two weight matrices in rotation (2 x 1.04 GB); bytes = weights and hidden states once")
+
+        def call_lm_kl(i, hs=hs, ws=ws):
+            dd.lm_head_verify(hs[(i + 1) % 2], ws[(i + 1) % 2], hs[i % 2], ws[i % 2], tokens, flags, K_, 0.5, 32, 0,
+                              out_tokens=ot, out_mask=om, out_score=osc)
+        record(name + ", KL (both heads)", "dd_lm_head_verify", dict(B=B, P=P, K=K, V=V, mode="KL", k=32), call_lm_kl, 2,
+               4.0 * B * P * K * V, 2.0 * (V * K * 2 + B * P * K * 2), "tensor",
+               note="the two matrices serve as drafter and verifier, roles swapped every call")
         del hs, ws
     assert dd.verify_status() == 0
     return out

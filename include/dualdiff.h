@@ -131,22 +131,25 @@ int dd_unmask(const void *logits, const int32_t *tokens, const uint8_t *mask_fla
               int B, int P, int V, void *stream);
 
 /*
- * The verifier's language-model head fused with the verification algorithm (Algorithm 1,
- * verification phase: p_V(. | x^D) is computed "for all positions" and handed to A(p_D, p_V, x^D);
- * Section 3.1).  Instead of logits the caller passes the verifier's last hidden states and its output
- * embedding:
- *     logits[b,i,x] = sum_j verifier_hidden[b,i,j] * verifier_weight[x,j]
+ * The language-model heads fused with the verification algorithm (Algorithm 1, verification
+ * phase: p_V(. | x^D) is computed "for all positions" and handed to A(p_D, p_V, x^D); Section 3.1).
+ * Instead of logits the caller passes last hidden states and output embeddings:
+ *     verifier logits[b,i,x] = sum_j verifier_hidden[b,i,j] * verifier_weight[x,j]
+ *     drafter  logits[b,i,x] = sum_j drafter_hidden[b,i,j]  * drafter_weight[x,j]     (DD_MODE_KL only)
  * (fp32 accumulation of bf16 products on the tensor cores, never rounded to bf16, never stored), and
- * the call gives what dd_verify gives on those logits in the modes that need the verifier only:
- * DD_MODE_TRUST and DD_MODE_CONF, with DD_FLAG_PROBABILISTIC / DD_FLAG_EMIT_DRAFTER as there.
- * DD_MODE_KL returns DD_ERR_UNSUPPORTED (the drafter's head is not fused).
- * verifier_hidden: [B,P,K] bf16; verifier_weight: [V,K] bf16 (row x = output embedding of token x);
- * both contiguous, K innermost, 16-byte aligned.  The other arguments, outputs, scratch and errors
- * are dd_verify's.  The hidden states of positions with mask_flags == 0 are read (they share tiles
- * with their neighbours) but nothing is computed from them.
+ * the call gives what dd_verify gives on those logits, in every mode and with DD_FLAG_PROBABILISTIC /
+ * DD_FLAG_EMIT_DRAFTER as there.  DD_MODE_TRUST and DD_MODE_CONF need the verifier only: the drafter's
+ * pair is not read and may be NULL.  DD_MODE_KL (Eq. 4-5) needs both pairs (DD_ERR_INVALID_ARG if one
+ * is NULL); the drafter's distribution is then the one its head gives on the same positions.
+ * verifier_hidden, drafter_hidden: [B,P,K] bf16; verifier_weight, drafter_weight: [V,K] bf16 (row x =
+ * output embedding of token x); all contiguous, K innermost, 16-byte aligned, the same K for both
+ * models.  The other arguments, outputs, scratch and errors are dd_verify's.  The hidden states of
+ * positions with mask_flags == 0 are read (they share tiles with their neighbours) but nothing is
+ * computed from them.
  * Supported: K a multiple of 64; any V >= 1; P <= 8192.
  */
-int dd_lm_head_verify(const void *verifier_hidden, const void *verifier_weight,
+int dd_lm_head_verify(const void *drafter_hidden, const void *drafter_weight,
+                      const void *verifier_hidden, const void *verifier_weight,
                       const int32_t *tokens, const uint8_t *mask_flags,
                       int mode, float tau, int k, uint64_t seed,
                       int32_t *out_tokens, uint8_t *out_mask, float *out_score,

@@ -69,7 +69,7 @@ def lib() -> ctypes.CDLL:
         L.dd_verify_workspace_bytes.restype = ctypes.c_size_t
         L.dd_launch_count.argtypes = []
         L.dd_launch_count.restype = u64
-        L.dd_lm_head_verify.argtypes = [vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.dd_lm_head_verify.argtypes = [vp, vp, vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, i32, vp]
         L.dd_lm_head_verify.restype = i32
         L.dd_clear_status.argtypes = []
         L.dd_clear_status.restype = i32
@@ -200,15 +200,20 @@ def verify(drafter_logits, verifier_logits, tokens, mask_flags, mode, tau, k, se
     return out_tokens, out_mask, out_score
 
 
-def lm_head_verify(verifier_hidden, verifier_weight, tokens, mask_flags, mode, tau, k, seed,
-                   out_tokens=None, out_mask=None, out_score=None, stream=None):
-    """dd_lm_head_verify: the verifier's language-model head fused with the verification algorithm.
+def lm_head_verify(drafter_hidden, drafter_weight, verifier_hidden, verifier_weight, tokens, mask_flags,
+                   mode, tau, k, seed, out_tokens=None, out_mask=None, out_score=None, stream=None):
+    """dd_lm_head_verify: the language-model heads fused with the verification algorithm.
 
-    verifier_hidden [B,P,K], verifier_weight [V,K]: torch.bfloat16 device tensors.
+    verifier_hidden [B,P,K], verifier_weight [V,K]: torch.bfloat16 device tensors; drafter_hidden,
+    drafter_weight: the same shapes, or None in the modes that need the verifier only.
     Returns (out_tokens int32 [B,P], out_mask uint8 [B,P], out_score float32 [B,P])."""
     import torch
     B, P, K = verifier_hidden.shape
     V = verifier_weight.shape[0]
+    if drafter_hidden is not None:
+        _require(drafter_hidden, torch.bfloat16, (B, P, K), True, "drafter_hidden")
+    if drafter_weight is not None:
+        _require(drafter_weight, torch.bfloat16, (V, K), True, "drafter_weight")
     _require(verifier_hidden, torch.bfloat16, (B, P, K), True, "verifier_hidden")
     _require(verifier_weight, torch.bfloat16, (V, K), True, "verifier_weight")
     _require(tokens, torch.int32, (B, P), True, "tokens")
@@ -223,7 +228,8 @@ def lm_head_verify(verifier_hidden, verifier_weight, tokens, mask_flags, mode, t
     _require(out_tokens, torch.int32, (B, P), True, "out_tokens")
     _require(out_mask, torch.uint8, (B, P), True, "out_mask")
     _require(out_score, torch.float32, (B, P), True, "out_score")
-    _check(lib().dd_lm_head_verify(_ptr(verifier_hidden), _ptr(verifier_weight), _ptr(tokens), _ptr(mask_flags),
+    _check(lib().dd_lm_head_verify(_ptr(drafter_hidden), _ptr(drafter_weight), _ptr(verifier_hidden),
+                                   _ptr(verifier_weight), _ptr(tokens), _ptr(mask_flags),
                                    int(mode), float(tau), int(k), int(seed) & 0xFFFFFFFFFFFFFFFF,
                                    _ptr(out_tokens), _ptr(out_mask), _ptr(out_score), B, P, K, V, _stream_ptr(stream)))
     return out_tokens, out_mask, out_score

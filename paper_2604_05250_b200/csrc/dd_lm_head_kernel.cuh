@@ -1,19 +1,25 @@
-// Language-model head fused with the verification algorithm (Algorithm 1, verification phase:
+// Language-model heads fused with the verification algorithm (Algorithm 1, verification phase:
 // the verifier's distribution p_V(. | x^D) "for all positions" goes straight into A(p_D, p_V, x^D)).
 //
 // logits[t, x] = sum_k hidden[t, k] * weight[x, k] is a [rows, K] x [K, V] product whose result,
 // 253 KB per position at the LLaDA vocabulary, is only ever reduced: per row its maximum, the
-// lowest index of the maximum and the softmax normaliser (Eq. 7).  The kernel therefore keeps the
-// product in tensor memory and never stores a logit: a persistent CTA takes work items of
-// 256 rows x N vocabulary entries (N <= 256), accumulates them with tcgen05 MMAs (two
-// accumulators of 128 rows, fp32) from operand tiles that a TMA producer streams through a
-// three-stage ring, and its epilogue warps turn every accumulator row into one partial
-// (maximum, first index, sum 2^(l*log2e - M)) of the same form as the streaming kernel's chunk
-// partials.  Partials go through the same global table, row counters, fp64 row fold and decision
-// stage as dd_verify's, with "chunk" = vocabulary tile.
+// lowest index of the maximum and the softmax normaliser (Eq. 7), and in the KL mode the sums of
+// Eq. 4-5 over the drafter's logits, which are a second product of the same shape.  The kernel
+// therefore keeps the products in tensor memory and never stores a logit: a persistent CTA takes
+// work items of 256 rows x N vocabulary entries, accumulates them with tcgen05 MMAs (accumulators
+// of 128 rows, fp32) from operand tiles that a TMA producer streams through a three-stage ring,
+// and its epilogue warps turn every accumulator row into one partial (maximum, first index,
+// sum 2^(l*log2e - M); KL: also the drafter's maximum, sum and the weighted logit differences) of
+// the same form as the streaming kernel's chunk partials.  Partials go through the same global
+// table, row counters, fp64 row fold and decision stage as dd_verify's, with "chunk" = vocabulary
+// tile.
 //
-//   warps 0-3   epilogue of accumulator 0 (thread = row = tensor-memory lane)
-//   warps 4-7   epilogue of accumulator 1
+// Tensor memory (512 columns): TRUST/CONF, N <= 256: the verifier's two accumulators at columns 0
+// and 256.  KL, N <= 128: the drafter's at 0 and 128, the verifier's at 256 and 384; a work item
+// runs the k loop over the drafter's operands first, then over the verifier's.
+//
+//   warps 0-3   epilogue of rows 0-127 of the item (thread = row = tensor-memory lane)
+//   warps 4-7   epilogue of rows 128-255
 //   warp  8     one thread feeds the ring: per 64-wide k-step the two 128-row tiles of the hidden
 //               states and the N-row tile of the weights (2-D tensor maps, 128-byte swizzle, rows
 //               past the end read as zero; no multicast)
@@ -38,7 +44,7 @@ constexpr int kRowsPerItem = 256;          // two accumulators of 128 rows
 constexpr int kBlockK = 64;                // one 128-byte swizzled box per k-step
 constexpr int kStages = 3;
 constexpr int kMaxN = 256;
-constexpr uint32_t kTmemCols = 512;        // accumulator 0 in columns [0, N), accumulator 1 in [256, 256 + N)
+constexpr uint32_t kTmemCols = 512;        // see the layout above
 constexpr int kATileBytes = 128 * kBlockK * 2;                        // 16 KB: 128 rows x 64 bf16
 constexpr int kStageBytes = 2 * kATileBytes + kMaxN * kBlockK * 2;    // 64 KB
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
@@ -46,7 +52,7 @@ constexpr unsigned kErrLmFull = 0xC00, kErrLmEmpty = 0xD00, kErrLmAcc = 0xE00;
 
 struct LmParams {
     int rows, K, V;            // rows = B * P
-    int N;                     // vocabulary entries per work item (a multiple of 32, <= 256)
+    int N;                     // vocabulary entries per work item (a multiple of 32, <= 256; KL: <= 128)
     int n_tiles;               // ceil(V / N): the "chunks" of a row
     int row_blocks;            // ceil(rows / 256)
 };
@@ -55,13 +61,14 @@ struct LmParams {
 // 1 = a flagged row's partial, 0 = an unflagged row, reported to its sequence once, -1 = nothing).
 // One fence for the batch, one count per row; rows whose last tile this was are folded (fp64, tile
 // order) and reported; the warp that completes a sequence decides it.
+template <bool KL>
 __device__ __forceinline__ void publish_rows(const ddv::VerifyParams &p, const ddv::Partial &c, int row, int tile, int kind)
 {
     const unsigned full = 0xFFFFFFFFu;
     if (kind == 1) {
         ddv::Partial *dst = p.partials + (size_t)row * p.nchunks + tile;
-        __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), 0.f));
-        __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(0.f, 0.f, 0.f, 0.f));
+        __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d));
+        __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(c.s_d, c.t, 0.f, 0.f));
     }
     __threadfence();
     bool last = false;
@@ -70,7 +77,7 @@ __device__ __forceinline__ void publish_rows(const ddv::VerifyParams &p, const d
     while (todo) {
         const int src = __ffs(todo) - 1;
         todo &= todo - 1;
-        ddv::fold_row<false>(p, __shfl_sync(full, row, src), nullptr);
+        ddv::fold_row<KL>(p, __shfl_sync(full, row, src), nullptr);
     }
     todo = __ballot_sync(full, kind == 0);
     while (todo) {
@@ -81,7 +88,11 @@ __device__ __forceinline__ void publish_rows(const ddv::VerifyParams &p, const d
 }
 
 // Epilogue warps: every accumulator row becomes one partial.  Columns are visited in index order
-// with a strict comparison, so the index kept is the lowest index of the maximum.
+// with a strict comparison, so the index kept is the lowest index of the maximum.  KL (Eq. 4-5):
+// the drafter's accumulator is read beside the verifier's, and the row also keeps the drafter's
+// running maximum m_d, s_d = sum 2^(d*log2e - M_d) and t = sum 2^(d*log2e - M_d) * (d - v), both
+// rescaled whenever the maximum moves.
+template <bool KL>
 __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyParams &p, uint32_t tmem,
                                          uint32_t bar_acc_full, uint32_t bar_acc_empty,
                                          volatile uint32_t *abort_flag, int n_items)
@@ -89,7 +100,8 @@ __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyPar
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int acc = warp >> 2;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;          // this warp's 32 tensor-memory lanes
-    const uint32_t tacc = tmem + lane_off + (uint32_t)acc * 256u;
+    const uint32_t tacc = tmem + lane_off + (KL ? 256u + (uint32_t)acc * 128u : (uint32_t)acc * 256u);   // verifier
+    const uint32_t dacc = tmem + lane_off + (uint32_t)acc * 128u;                                          // drafter (KL)
     uint32_t n_done = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_done) {
         const int tile = item / q.row_blocks, rb = item - tile * q.row_blocks;
@@ -111,10 +123,12 @@ __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyPar
         }
         tc_fence_after();
         float m = -INFINITY, M = -INFINITY, s = 0.f;
+        float m_d = -INFINITY, M_d = -INFINITY, s_d = 0.f, t = 0.f;
         int idx = 0x7FFFFFFF;
         for (int cb = 0; cb < q.N / 32; ++cb) {
-            uint32_t r[32];
+            uint32_t r[32], rd[32];              // rd: the drafter's logits, KL only
             tmem_ld32(tacc + cb * 32, r);
+            if constexpr (KL) tmem_ld32(dacc + cb * 32, rd);
             tmem_wait_ld();
             const int valid = q.V - (col0 + cb * 32);                 // columns of this group that exist
             if (valid <= 0) break;
@@ -134,6 +148,26 @@ __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyPar
 #pragma unroll
             for (int i = 0; i < 32; ++i)
                 if (i < valid) s += ddv::ex2_approx(fmaf(__uint_as_float(r[i]), ddv::kLog2e, -M));
+            if constexpr (KL) {
+                float cd = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < valid) cd = fmaxf(cd, __uint_as_float(rd[i]));
+                if (cd > m_d) {
+                    const float M_new = cd * ddv::kLog2e;
+                    const float f = ddv::rescale_factor(M_d, M_new);
+                    s_d *= f; t *= f;
+                    m_d = cd; M_d = M_new;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < valid) {
+                        const float d = __uint_as_float(rd[i]);
+                        const float e = ddv::ex2_approx(fmaf(d, ddv::kLog2e, -M_d));
+                        s_d += e;
+                        t = fmaf(e, d - __uint_as_float(r[i]), t);
+                    }
+            }
         }
         // both accumulators may be overwritten once every epilogue warp has read its lanes
         tc_fence_before();
@@ -142,16 +176,21 @@ __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyPar
 
         ddv::Partial c;
         c.m_v = m; c.s_v = s; c.idx = idx;
-        c.m_d = 0.f; c.s_d = 0.f; c.t = 0.f; c.pad0 = c.pad1 = 0.f;
+        c.m_d = KL ? m_d : 0.f; c.s_d = s_d; c.t = t; c.pad0 = c.pad1 = 0.f;
         int kind = -1;
         if (row < q.rows) kind = p.flags[row] ? 1 : (tile == 0 ? 0 : -1);
-        publish_rows(p, c, min(row, q.rows - 1), tile, kind);
+        publish_rows<KL>(p, c, min(row, q.rows - 1), tile, kind);
     }
 }
 
-template <int kDummy>
+// KL: every work item runs the k loop twice, first over the drafter's hidden states and weights
+// into accumulators [0,N) and [128,128+N), then over the verifier's into [256,..) and [384,..)
+// (N <= 128); the epilogue reads both.  Otherwise only the verifier's maps are used and the
+// accumulators are [0,N) and [256,256+N) (N <= 256).
+template <bool KL>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w,
+               const __grid_constant__ CUtensorMap tm_hd, const __grid_constant__ CUtensorMap tm_wd,
                const LmParams q, const ddv::VerifyParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -171,6 +210,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__
 
     if (tid == 0) {
         prefetch_tmap(&tm_h); prefetch_tmap(&tm_w);
+        if (KL) { prefetch_tmap(&tm_hd); prefetch_tmap(&tm_wd); }
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         mbar_init(bar_acc_empty, kEpilogueWarps);
@@ -206,15 +246,18 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__
             const int tile = item / q.row_blocks, rb = item - tile * q.row_blocks;
             const int row0 = rb * kRowsPerItem, col0 = tile * q.N;
             bool ok = true;
-            for (int ks = 0; ks < k_steps; ++ks, ++step) {
+            for (int ks2 = 0; ks2 < (KL ? 2 : 1) * k_steps; ++ks2, ++step) {
                 const int s = step % kStages;
                 const uint32_t use = step / kStages;
                 if (use > 0 && !wait(bar_empty(s), (use - 1) & 1)) { give_up(kErrLmEmpty); ok = false; break; }
                 const uint32_t dst = smem_base + s * kStageBytes;
+                const bool drafter = KL && ks2 < k_steps;                 // the drafter's pass comes first
+                const int ks = ks2 < k_steps ? ks2 : ks2 - k_steps;
+                const CUtensorMap *mh = drafter ? &tm_hd : &tm_h, *mw = drafter ? &tm_wd : &tm_w;
                 mbar_expect_tx(bar_full(s), (uint32_t)(2 * kATileBytes + q.N * kBlockK * 2));
-                tma_load_2d(dst, &tm_h, bar_full(s), ks * kBlockK, row0);
-                tma_load_2d(dst + kATileBytes, &tm_h, bar_full(s), ks * kBlockK, row0 + 128);
-                tma_load_2d(dst + 2 * kATileBytes, &tm_w, bar_full(s), ks * kBlockK, col0);
+                tma_load_2d(dst, mh, bar_full(s), ks * kBlockK, row0);
+                tma_load_2d(dst + kATileBytes, mh, bar_full(s), ks * kBlockK, row0 + 128);
+                tma_load_2d(dst + 2 * kATileBytes, mw, bar_full(s), ks * kBlockK, col0);
             }
             if (!ok) break;
         }
@@ -227,18 +270,21 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__
             if (n_done > 0 && !wait(bar_acc_empty, (n_done - 1) & 1)) { give_up(kErrLmAcc); break; }
             tc_fence_after();
             bool ok = true;
-            for (int ks = 0; ks < k_steps; ++ks, ++step) {
+            for (int ks2 = 0; ks2 < (KL ? 2 : 1) * k_steps; ++ks2, ++step) {
                 const int s = step % kStages;
                 if (!wait(bar_full(s), (step / kStages) & 1)) { give_up(kErrLmFull); ok = false; break; }
                 tc_fence_after();
+                const int ks = ks2 < k_steps ? ks2 : ks2 - k_steps;
+                // accumulator columns of this pass: see the layout above
+                const uint32_t acc0 = tmem + ((KL && ks2 >= k_steps) ? 256u : 0u), acc1 = acc0 + (KL ? 128u : 256u);
                 const uint32_t base = smem_base + s * kStageBytes;
                 const uint64_t a0 = smem_desc_sw128(base, 16, 1024), a1 = smem_desc_sw128(base + kATileBytes, 16, 1024);
                 const uint64_t b = smem_desc_sw128(base + 2 * kATileBytes, 16, 1024);
 #pragma unroll
                 for (int kk = 0; kk < kBlockK / 16; ++kk) {
                     const uint32_t off = (uint32_t)(kk * 32) >> 4;            // 16 bf16 = 32 bytes per MMA
-                    mma_ss(tmem, a0 + off, b + off, idesc, (ks > 0 || kk > 0));
-                    mma_ss(tmem + 256, a1 + off, b + off, idesc, (ks > 0 || kk > 0));
+                    mma_ss(acc0, a0 + off, b + off, idesc, (ks > 0 || kk > 0));
+                    mma_ss(acc1, a1 + off, b + off, idesc, (ks > 0 || kk > 0));
                 }
                 mma_commit(bar_empty(s));                                      // the stage is free once these have run
             }
@@ -246,7 +292,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__
             mma_commit(bar_acc_full);
         }
     } else if (warp < kEpilogueWarps) {
-        epilogue(q, p, tmem, bar_acc_full, bar_acc_empty, abort_flag, n_items);
+        epilogue<KL>(q, p, tmem, bar_acc_full, bar_acc_empty, abort_flag, n_items);
     }
 
     __syncwarp();

@@ -452,13 +452,13 @@ int make_matrix_tmap(CUtensorMap *m, const void *base, long n_rows, int K, int b
     return DD_OK;
 }
 
-// Vocabulary entries per work item: the multiple of 32 (at most 256) for which the slowest CTA
-// of `ctas` has least to do.
-int pick_tile_n(int V, long row_blocks, int ctas)
+// Vocabulary entries per work item: the multiple of 32 (at most `max_n`, at least half of it) for
+// which the slowest CTA of `ctas` has least to do.
+int pick_tile_n(int V, long row_blocks, int ctas, int max_n)
 {
-    int best = 256;
+    int best = max_n;
     long best_cost = -1;
-    for (int n = 256; n >= 128; n -= 32) {
+    for (int n = max_n; n >= max_n / 2; n -= 32) {
         const long items = ((V + n - 1) / n) * row_blocks;
         const long cost = ((items + ctas - 1) / ctas) * n;
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
@@ -468,7 +468,8 @@ int pick_tile_n(int V, long row_blocks, int ctas)
 
 }  // namespace
 
-extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifier_weight,
+extern "C" int dd_lm_head_verify(const void *drafter_hidden, const void *drafter_weight,
+                                 const void *verifier_hidden, const void *verifier_weight,
                                  const int32_t *tokens, const uint8_t *mask_flags,
                                  int mode, float tau, int k, uint64_t seed,
                                  int32_t *out_tokens, uint8_t *out_mask, float *out_score,
@@ -476,11 +477,14 @@ extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifi
 {
     if (!verifier_hidden || !verifier_weight) return DD_ERR_INVALID_ARG;
     if (K <= 0) return DD_ERR_INVALID_ARG;
-    int rc = check_args(nullptr, verifier_hidden, tokens, mask_flags, mode, tau, k, out_tokens, out_mask, B, P, V);
-    if (rc == DD_ERR_INVALID_ARG && (mode & 0xFF) == DD_MODE_KL) return DD_ERR_UNSUPPORTED;      // the drafter's head is not fused yet
+    const bool kl = (mode & 0xFF) == DD_MODE_KL;
+    if (kl && !drafter_weight) return DD_ERR_INVALID_ARG;
+    int rc = check_args(kl ? drafter_hidden : nullptr, verifier_hidden, tokens, mask_flags, mode, tau, k, out_tokens,
+                        out_mask, B, P, V);
     if (rc != DD_OK) return rc;
     if (K % ddlm::kBlockK != 0) return DD_ERR_UNSUPPORTED;
     if ((((uintptr_t)verifier_hidden | (uintptr_t)verifier_weight) & 15) != 0) return DD_ERR_UNSUPPORTED;
+    if (kl && (((uintptr_t)drafter_hidden | (uintptr_t)drafter_weight) & 15) != 0) return DD_ERR_UNSUPPORTED;
     const long rows = (long)B * P;
     const int sms = sm_count_of_current_device();
     if (sms < 0) return sms;
@@ -490,7 +494,7 @@ extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifi
     ddlm::LmParams q;
     q.rows = (int)rows; q.K = K; q.V = V;
     q.row_blocks = (int)((rows + ddlm::kRowsPerItem - 1) / ddlm::kRowsPerItem);
-    q.N = pick_tile_n(V, q.row_blocks, sms);
+    q.N = pick_tile_n(V, q.row_blocks, sms, kl ? ddlm::kMaxN / 2 : ddlm::kMaxN);
     q.n_tiles = (V + q.N - 1) / q.N;
     if (rows * q.n_tiles >= (1L << 31) - (1L << 24)) return DD_ERR_UNSUPPORTED;
 
@@ -516,9 +520,14 @@ extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifi
     p.partials = (Partial *)w;
     fill_params(p, nullptr, nullptr, tokens, mask_flags, mode, tau, k, seed, out_tokens, out_mask, out_score, B, P, V);
 
-    CUtensorMap tm_h, tm_w;
+    CUtensorMap tm_h, tm_w, tm_hd, tm_wd;
     if ((rc = make_matrix_tmap(&tm_h, verifier_hidden, rows, K, 128)) != DD_OK) return rc;
     if ((rc = make_matrix_tmap(&tm_w, verifier_weight, V, K, q.N)) != DD_OK) return rc;
+    tm_hd = tm_h; tm_wd = tm_w;                    // not read outside the KL mode
+    if (kl) {
+        if ((rc = make_matrix_tmap(&tm_hd, drafter_hidden, rows, K, 128)) != DD_OK) return rc;
+        if ((rc = make_matrix_tmap(&tm_wd, drafter_weight, V, K, q.N)) != DD_OK) return rc;
+    }
 
     int dev = 0;
     DD_CUDA_TRY(cudaGetDevice(&dev));
@@ -526,14 +535,19 @@ extern "C" int dd_lm_head_verify(const void *verifier_hidden, const void *verifi
         static bool attr_done[64] = {};
         std::lock_guard<std::mutex> lock(g_mu);
         if (!attr_done[dev]) {
-            DD_CUDA_TRY(cudaFuncSetAttribute(ddlm::lm_head_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            DD_CUDA_TRY(cudaFuncSetAttribute(ddlm::lm_head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             ddlm::kSmemBytes));
+            DD_CUDA_TRY(cudaFuncSetAttribute(ddlm::lm_head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              ddlm::kSmemBytes));
             attr_done[dev] = true;
         }
     }
     const long items = (long)q.n_tiles * q.row_blocks;
     const unsigned grid = (unsigned)(items < ctas ? items : ctas);
-    ddlm::lm_head_kernel<0><<<grid, ddlm::kThreads, ddlm::kSmemBytes, (cudaStream_t)stream>>>(tm_h, tm_w, q, p);
+    if (kl)
+        ddlm::lm_head_kernel<true><<<grid, ddlm::kThreads, ddlm::kSmemBytes, (cudaStream_t)stream>>>(tm_h, tm_w, tm_hd, tm_wd, q, p);
+    else
+        ddlm::lm_head_kernel<false><<<grid, ddlm::kThreads, ddlm::kSmemBytes, (cudaStream_t)stream>>>(tm_h, tm_w, tm_hd, tm_wd, q, p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
     return DD_OK;

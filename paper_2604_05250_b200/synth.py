@@ -172,3 +172,34 @@ def lm_head_inputs(B, P, K, V, flagged, seed, bump=8.0):
     for b in range(B):
         flags[b, np.sort(rng.choice(P, size=counts[b], replace=False))] = 1
     return f32_to_bf16_bits(hidden), f32_to_bf16_bits(weight), tokens, flags
+
+
+def lm_head_pair_inputs(B, P, K, V, flagged, err, seed, bump=8.0):
+    """Both models' last hidden states and output embeddings, for the KL mode from hidden states.
+    The verifier's pair is lm_head_inputs' (same seed, same values).  The drafter has an embedding
+    of its own, the verifier's plus N(0, (0.1 * 2 / sqrt(K))^2) per entry; on a (1 - err) share of
+    the positions its hidden state is the verifier's plus N(0, 0.25^2) per entry (logits that
+    differ by about N(0, 0.5^2), as in verify_inputs) and the token is the position's hot token,
+    on the rest it is an independent N(0, 1) vector (no hot token) and the token is random.
+
+    Returns (drafter_hidden, drafter_weight, verifier_hidden, verifier_weight: uint16 bf16 bits,
+    tokens i32 [B,P], flags u8 [B,P])."""
+    rng = np.random.default_rng([int(seed), 0x1E4D])
+    counts = flag_counts(B, P, flagged, rng)
+    weight = rng.standard_normal((V, K), dtype=np.float32)
+    weight *= np.float32(2.0 / np.sqrt(K))
+    hidden = rng.standard_normal((B, P, K), dtype=np.float32)
+    hot = rng.integers(0, V, size=(B, P))
+    hidden += np.float32(bump / 4.0) * weight[hot]
+    tokens = rng.integers(0, V, size=(B, P)).astype(np.int32)
+    flags = np.zeros((B, P), dtype=np.uint8)
+    for b in range(B):
+        flags[b, np.sort(rng.choice(P, size=counts[b], replace=False))] = 1
+    # everything above draws what lm_head_inputs draws, in its order; the drafter comes after
+    weight_d = weight + np.float32(0.2 / np.sqrt(K)) * rng.standard_normal((V, K), dtype=np.float32)
+    wrong = rng.random((B, P)) < err
+    hidden_d = hidden + np.float32(0.25) * rng.standard_normal((B, P, K), dtype=np.float32)
+    hidden_d[wrong] = rng.standard_normal((int(wrong.sum()), K), dtype=np.float32)
+    tokens = np.where(wrong, tokens, hot).astype(np.int32)
+    return (f32_to_bf16_bits(hidden_d), f32_to_bf16_bits(weight_d), f32_to_bf16_bits(hidden),
+            f32_to_bf16_bits(weight), tokens, flags)

@@ -45,12 +45,12 @@ def check_attention(gpu_out_f64, oracle_out):
     return float(diff.max()), float(diff.mean())
 
 
-def check_verify(gpu_tokens, gpu_mask, gpu_score, ref, flags, tokens_in):
+def check_verify(gpu_tokens, gpu_mask, gpu_score, ref, flags, tokens_in, score_abs=SCORE_ABS_FLOOR):
     """ref: dict from oracle.verify; gpu_*: numpy arrays."""
     flags = flags.astype(bool)
     exempt = ref["exempt"].astype(bool)
     o_score = ref["out_score"]
-    tol = np.maximum(SCORE_REL * np.abs(o_score), SCORE_ABS_FLOOR)
+    tol = np.maximum(SCORE_REL * np.abs(o_score), score_abs)
     bad = np.abs(gpu_score.astype(np.float64) - o_score) > tol
     assert not bad.any(), (f"{bad.sum()} scores out of tolerance; worst "
                            f"{np.abs(gpu_score - o_score).max():.3e}")
