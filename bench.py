@@ -322,6 +322,11 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
     window = 0.1 if quick else 0.25
 
     def record(name, op, shape, enqueue_one, n_sets, flops, nbytes, bound, note=None):
+        # The inputs were drawn on the default stream and the launches go to `stream`: everything
+        # queued so far has to finish first, both for the inputs themselves and because the caching
+        # allocator may already have handed a generator's temporary (still to be read by a queued
+        # kernel) to one of the output tensors.
+        torch.cuda.synchronize()
         # a graph of enough launches to last a few milliseconds, replayed over the window
         with torch.cuda.stream(stream):
             for i in range(3):
@@ -574,6 +579,7 @@ def run_ours(args):
         verify_call(i)
 
     stream = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize()               # the inputs were copied on the default stream
     sampler.start()
     with torch.cuda.stream(stream):
         for i in range(W):
@@ -736,6 +742,39 @@ def run_ours(args):
     return 0
 
 
+def print_tables(path):
+    """Markdown tables of a stored JSON line of this program (the last line of `path` that is one):
+    the headline step, its two kernels, and every entry of `other_configs`."""
+    with open(path) as f:
+        d = json.loads([ln for ln in f if ln.startswith("{")][-1])
+    ck, lat = d["clocks"], d["latency"]
+    print(f"Headline ({d['config']['workload']}): {1e3 * d['value']:.2f} us per step (median; "
+          f"p10 {1e3 * lat['p10_ms']:.2f}, p90 {1e3 * lat['p90_ms']:.2f}; eager launches "
+          f"{1e3 * lat['eager_median_ms']:.2f} us); e2e {d['e2e']['value']:.3f} ms; SM clock median "
+          f"{ck['sm_mhz']} of {ck['sm_max_mhz']} MHz, reasons {ck['reasons']}\n")
+    print("| kernel | us | achieved | of measured | of nominal |")
+    print("|---|---|---|---|---|")
+    for name, k in d["kernels"].items():
+        if "tflops" in k:
+            print(f"| {name} | {1e3 * k['ms']:.2f} | {k['tflops']:.0f} TFLOP/s | {k['frac_of_measured']:.3f} (burst) | "
+                  f"{k['frac_of_nominal_2250']:.3f} of 2250 |")
+        else:
+            print(f"| {name} | {1e3 * k['ms']:.2f} | {k['gbs']:.0f} GB/s | {k['frac_of_measured']:.3f} | "
+                  f"{k['frac_of_nominal_8000']:.3f} of 8000 |")
+    print("\n| workload | entry point | us (median) | p10 / p90 | achieved | of measured | of nominal | SM MHz (reasons) |")
+    print("|---|---|---|---|---|---|---|---|")
+    for e in d.get("other_configs", []):
+        if e["bound"] == "tensor":
+            perf = (f"{e['tflops']:.0f} TFLOP/s | {e['frac_of_measured_burst']:.3f} burst, "
+                    f"{e['frac_of_measured_sustained']:.3f} sustained | {e['frac_of_nominal_2250']:.3f}")
+        else:
+            perf = f"{e['gbs']:.0f} GB/s | {e['frac_of_measured_hbm']:.3f} | {e['frac_of_nominal_8000']:.3f}"
+        c = e["clocks"]
+        print(f"| {e['name']} | {e['op']} | {1e3 * e['ms']:.1f} | {1e3 * e['p10']:.1f} / {1e3 * e['p90']:.1f} | {perf} | "
+              f"{c['sm_mhz']} ({', '.join(c['reasons']) or 'none'}) |")
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -746,7 +785,11 @@ def main():
     ap.add_argument("--quick", action="store_true", help="shorter timing windows for the other configurations")
     ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1"],
                     help="launch K steps (or calls on one of two other shapes) eagerly and exit: for profilers")
+    ap.add_argument("--tables", metavar="FILE", default=None,
+                    help="print markdown tables of a stored JSON line of this program and exit (no GPU needed)")
     args = ap.parse_args()
+    if args.tables:
+        return print_tables(args.tables)
     if args.steps < 1:
         ap.error("--steps must be >= 1")
     return run_reference(args) if args.impl == "reference" else run_ours(args)
