@@ -495,6 +495,26 @@ def run_eager_other(dd, which, K, W):
         def call(i):
             q, k, v = sets[i % 2]
             dd.block_attention(q, k, v, out=o)
+    elif which in ("lm_head_small", "lm_head_small_kl"):
+        # a small case of the fused head: 256 rows, K = 4096, a 32000-entry vocabulary (262 MB of
+        # weights per matrix: larger than the L2, under 1 GB on the device)
+        B, P, K_, V = 1, 256, 4096, 32000
+        hs = [torch.randn(B, P, K_, device=dev, generator=gen).to(torch.bfloat16) for _ in range(2)]
+        ws = [(torch.randn(V, K_, device=dev, generator=gen) * (2.0 / K_ ** 0.5)).to(torch.bfloat16) for _ in range(2)]
+        tokens = torch.zeros(B, P, device=dev, dtype=torch.int32)
+        flags = torch.ones(B, P, device=dev, dtype=torch.uint8)
+        ot, om = torch.empty_like(tokens), torch.empty_like(flags)
+        oc = torch.empty(B, P, device=dev, dtype=torch.float32)
+        kl = which.endswith("_kl")
+        name = f"dd_lm_head_verify {'KL' if kl else 'CONF'} on hidden [{B},{P},{K_}], weights [{V},{K_}]"
+
+        def call(i):
+            if kl:
+                dd.lm_head_verify(hs[(i + 1) % 2], ws[(i + 1) % 2], hs[i % 2], ws[i % 2], tokens, flags, synth.MODE_KL,
+                                  0.5, 32, 0, out_tokens=ot, out_mask=om, out_score=oc)
+            else:
+                dd.lm_head_verify(None, None, hs[i % 2], ws[i % 2], tokens, flags, synth.MODE_CONF, 0.5, 32, 0,
+                                  out_tokens=ot, out_mask=om, out_score=oc)
     else:
         B, P, V = VER["B"], VER["P"], VER["V"]
         sets = [device_logits(B, P, V, 0.1, gen, False)[1] for _ in range(5)]
@@ -540,7 +560,7 @@ def run_ours(args):
     dd.lib()
 
     K, W = args.steps, max(3, args.warmup)
-    if args.eager_only in ("drafter_block", "unmask_cfg1"):
+    if args.eager_only in ("drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl"):
         return run_eager_other(dd, args.eager_only, K, W)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
 
@@ -783,8 +803,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-other-configs", action="store_true", help="time the headline step only")
     ap.add_argument("--quick", action="store_true", help="shorter timing windows for the other configurations")
-    ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1"],
-                    help="launch K steps (or calls on one of two other shapes) eagerly and exit: for profilers")
+    ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl"],
+                    help="launch K steps (or calls on one of the other shapes) eagerly and exit: for profilers")
     ap.add_argument("--tables", metavar="FILE", default=None,
                     help="print markdown tables of a stored JSON line of this program and exit (no GPU needed)")
     args = ap.parse_args()
