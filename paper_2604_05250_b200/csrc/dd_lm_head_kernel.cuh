@@ -10,9 +10,10 @@
 // of 128 rows, fp32) from operand tiles that a TMA producer streams through a three-stage ring,
 // and its epilogue warps turn every accumulator row into one partial (maximum, first index,
 // sum 2^(l*log2e - M); KL: also the drafter's maximum, sum and the weighted logit differences) of
-// the same form as the streaming kernel's chunk partials.  Partials go through the same global
-// table, row counters, fp64 row fold and decision stage as dd_verify's, with "chunk" = vocabulary
-// tile.
+// the same form as the streaming kernel's chunk partials, stored in the same global table ("chunk"
+// = vocabulary tile).  A second, small kernel behind it on the stream (lm_head_fold_kernel) folds
+// every flagged row's partials in fp64 with the streaming kernel's fold and runs dd_verify's
+// decision stage per sequence.
 //
 // Tensor memory (512 columns): TRUST/CONF, N <= 256: the verifier's two accumulators at columns 0
 // and 256.  KL, N <= 128: the drafter's at 0 and 128, the verifier's at 256 and 384; a work item
@@ -57,33 +58,60 @@ struct LmParams {
     int row_blocks;            // ceil(rows / 256)
 };
 
-// Up to 32 rows' partials of one vocabulary tile (lane l holds row `row` and its partial; `kind`:
-// 1 = a flagged row's partial, 0 = an unflagged row, reported to its sequence once, -1 = nothing).
-// One fence for the batch, one count per row; rows whose last tile this was are folded (fp64, tile
-// order) and reported; the warp that completes a sequence decides it.
-template <bool KL>
-__device__ __forceinline__ void publish_rows(const ddv::VerifyParams &p, const ddv::Partial &c, int row, int tile, int kind)
+// One row's partial of one vocabulary tile into the global table.  Nothing else happens in this
+// kernel: rows are folded and sequences decided by lm_head_fold_kernel, launched behind it on the
+// same stream.  (Folding in here, by whichever warp stores a row's last tile, put every fold of the
+// launch on the one CTA that finishes last: all rows of a row block complete together, with the
+// last tile.  170 of 217 us on a 256-row, 143-tile problem were that CTA folding alone.)
+__device__ __forceinline__ void store_partial(const ddv::VerifyParams &p, const ddv::Partial &c, int row, int tile)
 {
-    const unsigned full = 0xFFFFFFFFu;
-    if (kind == 1) {
-        ddv::Partial *dst = p.partials + (size_t)row * p.nchunks + tile;
-        __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d));
-        __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(c.s_d, c.t, 0.f, 0.f));
+    ddv::Partial *dst = p.partials + (size_t)row * p.nchunks + tile;
+    __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d));
+    __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(c.s_d, c.t, 0.f, 0.f));
+}
+
+// n more rows of sequence b are accounted for (warp-level); the warp that accounts for the last
+// of the P rows decides the sequence.
+__device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int n)
+{
+    const int lane = threadIdx.x & 31;
+    int last = 0;
+    if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(p.seq_counter + b, (unsigned)n) + (unsigned)n == (unsigned)p.P;
     }
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
     __threadfence();
-    bool last = false;
-    if (kind == 1) last = atomicAdd(p.row_counter + row, 1u) == (unsigned)(p.nchunks - 1);
-    unsigned todo = __ballot_sync(full, last);
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        todo &= todo - 1;
-        ddv::fold_row<KL>(p, __shfl_sync(full, row, src), nullptr);
-    }
-    todo = __ballot_sync(full, kind == 0);
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        todo &= todo - 1;
-        ddv::row_done(p, __shfl_sync(full, row, src) / p.P, nullptr);
+    if (lane == 0) p.seq_counter[b] = 0u;      // ready for the next launch
+    ddv::decide_sequence(p, b, nullptr);
+}
+
+// Second launch of dd_lm_head_verify: one warp per row folds the row's tile partials (fp64, tile
+// order: the streaming kernel's fold) and stores score and argmax; one warp per sequence accounts
+// for the rows that are not flagged; the warp that accounts for a sequence's last row runs the
+// decision stage.  The partials were written by the previous kernel on the stream.
+constexpr int kFoldThreads = 128;
+template <bool KL>
+__global__ void __launch_bounds__(kFoldThreads) lm_head_fold_kernel(const ddv::VerifyParams p, int rows)
+{
+    const int w = blockIdx.x * (kFoldThreads / 32) + (threadIdx.x >> 5);     // rows first, then sequences
+    if (w < rows) {
+        if (!p.flags[w]) return;
+        float score;
+        int argmax;
+        ddv::fold_partials<KL>(p.partials + (size_t)w * p.nchunks, p.nchunks, score, argmax);
+        if ((threadIdx.x & 31) == 0) {
+            __stcg(p.row_score + w, score);
+            __stcg(p.row_argmax + w, argmax);
+        }
+        __syncwarp();
+        rows_done(p, w / p.P, 1);
+    } else {
+        const int b = w - rows;
+        if (b >= p.B) return;
+        const int unflagged = p.P - ddv::count_flagged(p, b);
+        if (unflagged > 0) rows_done(p, b, unflagged);
     }
 }
 
@@ -177,9 +205,7 @@ __device__ __forceinline__ void epilogue(const LmParams &q, const ddv::VerifyPar
         ddv::Partial c;
         c.m_v = m; c.s_v = s; c.idx = idx;
         c.m_d = KL ? m_d : 0.f; c.s_d = s_d; c.t = t; c.pad0 = c.pad1 = 0.f;
-        int kind = -1;
-        if (row < q.rows) kind = p.flags[row] ? 1 : (tile == 0 ? 0 : -1);
-        publish_rows<KL>(p, c, min(row, q.rows - 1), tile, kind);
+        if (row < q.rows && p.flags[row]) store_partial(p, c, row, tile);
     }
 }
 

@@ -550,6 +550,14 @@ extern "C" int dd_lm_head_verify(const void *drafter_hidden, const void *drafter
         ddlm::lm_head_kernel<false><<<grid, ddlm::kThreads, ddlm::kSmemBytes, (cudaStream_t)stream>>>(tm_h, tm_w, tm_hd, tm_wd, q, p);
     DD_CUDA_TRY(cudaGetLastError());
     dd::count_launch();
+    // one warp per row, then one per sequence
+    const unsigned fold_grid = (unsigned)((rows + B + ddlm::kFoldThreads / 32 - 1) / (ddlm::kFoldThreads / 32));
+    if (kl)
+        ddlm::lm_head_fold_kernel<true><<<fold_grid, ddlm::kFoldThreads, 0, (cudaStream_t)stream>>>(p, (int)rows);
+    else
+        ddlm::lm_head_fold_kernel<false><<<fold_grid, ddlm::kFoldThreads, 0, (cudaStream_t)stream>>>(p, (int)rows);
+    DD_CUDA_TRY(cudaGetLastError());
+    dd::count_launch();
     return DD_OK;
 }
 
