@@ -285,14 +285,19 @@ __device__ __noinline__ void fold_partials(const Partial *src, int n, float &sco
         if (om > bm_v || (om == bm_v && oi < bidx)) { bm_v = om; bidx = oi; }
         bm_d = fmaxf(bm_d, __shfl_xor_sync(0xFFFFFFFFu, bm_d, o));
     }
-    const float Mv = bm_v * kLog2e, Md = bm_d * kLog2e;
+    const float Mv = __fmul_rn(bm_v, kLog2e), Md = __fmul_rn(bm_d, kLog2e);
     double sv = 0.0, sd = 0.0, tt = 0.0;
     for (int ch = lane; ch < n; ch += 32) {
         const float4 a = ld_volatile16(src + ch);
         const float4 bq = ld_volatile16(reinterpret_cast<const float4 *>(src + ch) + 1);
-        sv += (double)a.y * exp2((double)(a.x * kLog2e) - (double)Mv);
+        // the factor that moves a chunk's sums to the row's reference point is a power of two with a
+        // fractional exponent: one ex2.approx (2^-22 relative, the accuracy of every term inside
+        // the chunk sums), not a double-precision exp2 (a long software routine on this path,
+        // which sits at the very end of a launch).  The product is rounded on its own (no fused
+        // multiply-add), as Mv and Md were: the maximum's chunk gets the factor 2^0 exactly.
+        sv += (double)a.y * (double)ex2_approx(__fmul_rn(a.x, kLog2e) - Mv);
         if (KL) {
-            const double f = exp2((double)(a.w * kLog2e) - (double)Md);
+            const double f = (double)ex2_approx(__fmul_rn(a.w, kLog2e) - Md);
             sd += (double)bq.x * f;
             tt += (double)bq.y * f;
         }
