@@ -145,7 +145,8 @@ int dd_unmask(const void *logits, const int32_t *tokens, const uint8_t *mask_fla
  * output embedding of token x); all contiguous, K innermost, 16-byte aligned, the same K for both
  * models.  The other arguments, outputs, scratch and errors are dd_verify's.  The hidden states of
  * positions with mask_flags == 0 are read (they share tiles with their neighbours) but nothing is
- * computed from them.
+ * computed from them.  Two kernels per call, in stream order: the products with their per-tile
+ * reductions, then a small one that combines the tiles of every row and decides the sequences.
  * Supported: K a multiple of 64; any V >= 1; P <= 8192.
  */
 int dd_lm_head_verify(const void *drafter_hidden, const void *drafter_weight,
