@@ -500,6 +500,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (warp == 0) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
+#include "dd_attention_persistent.cuh"
+
 // ---------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -571,6 +573,44 @@ int launch(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, 
     return DD_OK;
 }
 
+// The persistent kernel: one CTA per SM (or per item, if there are fewer).
+template <int D>
+int launch_persistent(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
+                      const AttnParams &p, int sms, cudaStream_t s)
+{
+    static bool attr_done[64] = {};
+    static std::mutex attr_mu;
+    int dev = 0;
+    DD_CUDA_TRY(cudaGetDevice(&dev));
+    const int smem = SmemP<D>::kTotal + 1024;
+    {
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+            DD_CUDA_TRY(cudaFuncSetAttribute(attention_persistent_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attr_done[dev] = true;
+        }
+    }
+    const long items = (long)p.BH * p.m_blocks;
+    const unsigned grid = (unsigned)(items < sms ? items : sms);
+    attention_persistent_kernel<D><<<grid, kThreads, smem, s>>>(tq, tk, tv, to, p);
+    DD_CUDA_TRY(cudaGetLastError());
+    dd::count_launch();
+    return DD_OK;
+}
+
+int sm_count(int *out)
+{
+    static int cached[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    DD_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < 0 || dev >= 64) return DD_ERR_UNSUPPORTED;
+    if (cached[dev] == 0) DD_CUDA_TRY(cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev));
+    *out = cached[dev];
+    return DD_OK;
+}
+
 int attention_impl(const void *q, const void *k, const void *v, void *out, int B, int H, int Nq, int Nkv, int D,
                    const int32_t *kv_len, int layout, float scale, void *stream)
 {
@@ -612,6 +652,13 @@ int attention_impl(const void *q, const void *k, const void *v, void *out, int B
     cudaStream_t s = (cudaStream_t)stream;
     const bool general = kv_len != nullptr || !head_major || Nq != Nkv;
     if (general) return D == 64 ? launch<64, true>(tq, tk, tv, to, p, s) : launch<128, true>(tq, tk, tv, to, p, s);
+    // Many short items (more than one per SM, at most sixteen key tiles each, two query tiles in
+    // every item): the persistent kernel overlaps each item's start and end with its neighbours.
+    int sms = 0;
+    if ((rc = sm_count(&sms)) != DD_OK) return rc;
+    const int nkv = (Nkv + kBlockN - 1) / kBlockN;
+    if (BH * m_blocks > sms && nkv <= 16 && (Nq - 1) % (kQTiles * kBlockM) >= kBlockM)
+        return D == 64 ? launch_persistent<64>(tq, tk, tv, to, p, sms, s) : launch_persistent<128>(tq, tk, tv, to, p, sms, s);
     return D == 64 ? launch<64, false>(tq, tk, tv, to, p, s) : launch<128, false>(tq, tk, tv, to, p, s);
 }
 
