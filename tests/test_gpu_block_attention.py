@@ -129,6 +129,43 @@ def test_square_case_equals_bidirectional_attention(dd):
             assert (a.float() - c.float()).abs().max().item() <= 4e-3
 
 
+# ---- the drafter's shape with more (batch, head) items than SMs, key counts differing from
+# sequence to sequence
+
+@pytest.mark.parametrize("layout", ["bhnd", "bnhd"])
+@pytest.mark.parametrize("D", [64, 128])
+def test_many_heads_ragged_keys(dd, oracle_mod, layout, D):
+    import torch
+    B, H, Nq, Nkv = 12, 16, 32, 600            # 192 items
+    assert B * H > torch.cuda.get_device_properties(0).multi_processor_count
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 61)
+    # no key, one key, one tile, one key more, an odd number of tiles, all keys; twice, so that
+    # consecutive items of a CTA differ in every way
+    kv_len = np.array([600, 0, 1, 128, 129, 300, 0, 0, 511, 257, 600, 64], dtype=np.int32)
+    junk = np.array([0x7FC0, 0x7F80, 0xFF80, 0xFFFF], dtype=np.uint16)       # NaN, +inf, -inf, NaN
+    for b in range(B):
+        n = Nkv - kv_len[b]
+        k[b, :, kv_len[b]:] = junk[np.arange(n * D).reshape(n, D) % 4]
+        v[b, :, kv_len[b]:] = junk[(np.arange(n * D).reshape(n, D) + 1) % 4]
+    ref = oracle_mod.block_attention(q, k, v, D ** -0.5, kv_len=kv_len)
+    assert np.isfinite(ref).all()
+    if layout == "bnhd":
+        q, k, v = (np.ascontiguousarray(a.transpose(0, 2, 1, 3)) for a in (q, k, v))
+        ref = np.ascontiguousarray(ref.transpose(0, 2, 1, 3))
+    got = run_gpu(dd, q, k, v, D ** -0.5, kv_len=kv_len, layout=layout)
+    check_attention(got, ref)
+    zero = got[[1, 6, 7]] if layout == "bhnd" else got[[1, 6, 7]]
+    assert (zero == 0).all()                        # sequences without keys: zero output
+
+
+@pytest.mark.parametrize("Nq,Nkv", [(1, 1), (128, 1024), (100, 130), (7, 4096)])
+def test_many_heads_shapes(dd, oracle_mod, Nq, Nkv):
+    B, H, D = 5, 32, 128                        # 160 items, no kv_len: every key counts
+    q, k, v = block_inputs(B, H, Nq, Nkv, D, 70 + Nq)
+    got = run_gpu(dd, q, k, v, D ** -0.5)
+    check_attention(got, oracle_mod.block_attention(q, k, v, D ** -0.5))
+
+
 def test_peaked_rows_with_planted_structure(dd, oracle_mod):
     q, k, v = block_inputs(1, 2, 128, 1536, 128, 44, planted=True)
     got = run_gpu(dd, q, k, v, 128 ** -0.5, kv_len=np.array([1500], dtype=np.int32))
