@@ -495,6 +495,15 @@ def run_eager_other(dd, which, K, W):
         def call(i):
             q, k, v = sets[i % 2]
             dd.block_attention(q, k, v, out=o)
+    elif which == "attention_cfg2":
+        B, H, N, D = 16, 32, 512, 128          # many short work items: the persistent attention kernel
+        sets = [tuple(torch.randn(B, H, N, D, device=dev, generator=gen).to(torch.bfloat16) for _ in range(3)) for _ in range(3)]
+        o = torch.empty(B, H, N, D, device=dev, dtype=torch.bfloat16)
+        name = f"dd_bidir_attention B={B} H={H} N={N} D={D}"
+
+        def call(i):
+            q, k, v = sets[i % 3]
+            dd.bidir_attention(q, k, v, out=o)
     elif which in ("lm_head_small", "lm_head_small_kl"):
         # a small case of the fused head: 256 rows, K = 4096, a 32000-entry vocabulary (262 MB of
         # weights per matrix: larger than the L2, under 1 GB on the device)
@@ -560,7 +569,7 @@ def run_ours(args):
     dd.lib()
 
     K, W = args.steps, max(3, args.warmup)
-    if args.eager_only in ("drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl"):
+    if args.eager_only in ("drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl", "attention_cfg2"):
         return run_eager_other(dd, args.eager_only, K, W)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
 
@@ -803,7 +812,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-other-configs", action="store_true", help="time the headline step only")
     ap.add_argument("--quick", action="store_true", help="shorter timing windows for the other configurations")
-    ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl"],
+    ap.add_argument("--eager-only", nargs="?", const="step", default=None, choices=["step", "drafter_block", "unmask_cfg1", "lm_head_small", "lm_head_small_kl", "attention_cfg2"],
                     help="launch K steps (or calls on one of the other shapes) eagerly and exit: for profilers")
     ap.add_argument("--tables", metavar="FILE", default=None,
                     help="print markdown tables of a stored JSON line of this program and exit (no GPU needed)")
