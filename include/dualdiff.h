@@ -132,7 +132,7 @@ int dd_unmask(const void *logits, const int32_t *tokens, const uint8_t *mask_fla
 
 /*
  * The language-model heads fused with the verification algorithm (Algorithm 1, verification
- * phase: p_V(. | x^D) is computed "for all positions" and handed to A(p_D, p_V, x^D); Section 3.1).
+ * phase: p_V(. | x^D) is computed at every position and handed to A(p_D, p_V, x^D); Section 3.1).
  * Instead of logits the caller passes last hidden states and output embeddings:
  *     verifier logits[b,i,x] = sum_j verifier_hidden[b,i,j] * verifier_weight[x,j]
  *     drafter  logits[b,i,x] = sum_j drafter_hidden[b,i,j]  * drafter_weight[x,j]     (DD_MODE_KL only)

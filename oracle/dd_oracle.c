@@ -489,9 +489,9 @@ void dd_oracle_lm_head(const uint16_t *hidden, const uint16_t *weight, const uin
 
 /* ------------------------------------------------------------------------ */
 /* Unmask(p, x): one confidence-based unmasking step of a masked diffusion
- * model (Algorithm 1, drafting phase; Section 2.1: "a subset of
- * high-confidence tokens are unmasked"; Section 2.3: all tokens above a
- * confidence threshold, rather than a fixed number per step).
+ * model (Algorithm 1, drafting phase; Section 2.1: each step reveals the
+ * masked positions the model is most sure of; Section 2.3: every position
+ * above a confidence threshold, rather than a fixed number per step).
  *
  * For every masked position i (flags = 1): p_i = softmax(logits_i),
  * a_i = argmax (lowest index), c_i = p_i(a_i).  Position i is unmasked iff

@@ -1,5 +1,5 @@
 // Language-model heads fused with the verification algorithm (Algorithm 1, verification phase:
-// the verifier's distribution p_V(. | x^D) "for all positions" goes straight into A(p_D, p_V, x^D)).
+// the verifier's distribution p_V(. | x^D) at every position goes straight into A(p_D, p_V, x^D)).
 //
 // logits[t, x] = sum_k hidden[t, k] * weight[x, k] is a [rows, K] x [K, V] product whose result,
 // 253 KB per position at the LLaDA vocabulary, is only ever reduced: per row its maximum, the
