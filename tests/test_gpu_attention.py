@@ -128,3 +128,51 @@ def test_bitwise_repeatability(dd):
     first = run_gpu(dd, q, k, v, 128 ** -0.5)
     for _ in range(3):
         assert np.array_equal(first, run_gpu(dd, q, k, v, 128 ** -0.5))
+
+
+# ---- more (head, 256-row block) work items than SMs, each with few key tiles: dd_bidir_attention
+# runs these on persistent CTAs that walk over several items
+
+@pytest.mark.parametrize("B,H,N,D", [(6, 32, 200, 64), (5, 32, 440, 128), (3, 64, 256, 128), (2, 96, 130, 64)])
+def test_many_short_items(dd, oracle_mod, B, H, N, D):
+    import torch
+    assert B * H * ((N + 255) // 256) > torch.cuda.get_device_properties(0).multi_processor_count
+    q, k, v = synth.attention_inputs(B, H, N, D, seed=1000 + N)
+    got = run_gpu(dd, q, k, v, D ** -0.5)
+    check_attention(got, oracle_mod.attention(q, k, v, D ** -0.5))
+
+
+def test_many_short_items_peaked_rows(dd, oracle_mod):
+    """Rows whose maximum outgrows the reference point they inherit: the accumulator in tensor
+    memory is rescaled in the middle of an item, on CTAs that carry their barriers' phases over
+    from the items before.  Same bits as one CTA per item (one sequence per call), and the first
+    heads of every sequence against the oracle."""
+    import torch
+    q, k, v = synth.attention_inputs(5, 32, 512, 128, seed=61, planted=True, strength=6.0)
+    tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
+    g = Guarded(tq.shape, torch.bfloat16)
+    whole = dd.bidir_attention(tq, tk, tv, out=g.view, scale=128 ** -0.5)
+    parts = torch.cat([dd.bidir_attention(tq[i:i + 1].contiguous(), tk[i:i + 1].contiguous(), tv[i:i + 1].contiguous(),
+                                          scale=128 ** -0.5) for i in range(5)], dim=0)
+    torch.cuda.synchronize()
+    assert dd.attention_status() == 0
+    g.check("attention output")
+    assert torch.equal(whole, parts)
+    sub = slice(0, 2)
+    ref = oracle_mod.attention(np.ascontiguousarray(q[:, sub]), np.ascontiguousarray(k[:, sub]),
+                               np.ascontiguousarray(v[:, sub]), 128 ** -0.5)
+    check_attention(bf16_tensor_to_f64(whole[:, sub]), ref)
+
+
+def test_many_short_items_match_one_item_per_cta(dd):
+    """The same 320 items in one call (persistent CTAs) and in four calls of 80 (one CTA per
+    item): the same arithmetic in the same order, so the same bits."""
+    import torch
+    q, k, v = synth.attention_inputs(1, 160, 512, 128, seed=62)
+    tq, tk, tv = (to_torch_bf16(x, "cuda") for x in (q, k, v))
+    whole = dd.bidir_attention(tq, tk, tv)
+    parts = [dd.bidir_attention(tq[:, i:i + 40].contiguous(), tk[:, i:i + 40].contiguous(), tv[:, i:i + 40].contiguous())
+             for i in range(0, 160, 40)]
+    torch.cuda.synchronize()
+    assert dd.attention_status() == 0
+    assert torch.equal(whole, torch.cat(parts, dim=1))
