@@ -343,6 +343,30 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const float inv = (!kBlock || nkv > 0) ? 1.f / l_run : 0.f;
                 const float w_own = scale_own * inv, w_other = scale_other * inv;
                 const uint32_t stage = sQ + g * kTileBytes + r * 128;
+                if constexpr (!kBlock) {
+                    // the whole accumulator row in one go: every load is in flight before the first is waited for
+                    uint32_t acc[D];
+#pragma unroll
+                    for (int cb = 0; cb < D / 32; ++cb)
+                        tmem_ld32(tO + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[cb * 32]));
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int cb = 0; cb < D / 32; ++cb) {
+                        const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[cb * 32 + i + 2 * h]) * inv,
+                                                                         __uint_as_float(acc[cb * 32 + i + 2 * h + 1]) * inv);
+                                w[h] = *reinterpret_cast<uint32_t *>(&v);
+                            }
+                            const int chunk = (cb % 2) * 4 + i / 8;         // 16-byte chunk of the 128-byte row
+                            st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                } else
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
                     uint32_t acc[32];

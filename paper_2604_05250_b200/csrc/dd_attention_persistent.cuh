@@ -163,24 +163,25 @@ attention_persistent_kernel(const __grid_constant__ CUtensorMap tm_q, const __gr
                 const int r = (warp & 3) * 32 + lane;
                 const float inv = 1.f / l_run;
                 const uint32_t stage = q_buf(par, g) + r * 128;
+                // the whole accumulator row in one go; once it is in registers the next item's first
+                // P V may overwrite the accumulator
+                uint32_t acc[D];
+#pragma unroll
+                for (int cb = 0; cb < D / 32; ++cb)
+                    tmem_ld32(tO + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[cb * 32]));
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar_o_free(g));
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
-                    uint32_t acc[32];
-                    tmem_ld32(tO + cb * 32, acc);
-                    tmem_wait_ld();
-                    if (cb == D / 32 - 1) {
-                        // the accumulator has been read: the next item's first P V may overwrite it
-                        tc_fence_before();
-                        mbar_arrive(bar_o_free(g));
-                    }
                     const uint32_t box = stage + (cb / 2) * kBoxBytes;
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint32_t w[4];
 #pragma unroll
                         for (int h = 0; h < 4; ++h) {
-                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * inv,
-                                                                     __uint_as_float(acc[i + 2 * h + 1]) * inv);
+                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[cb * 32 + i + 2 * h]) * inv,
+                                                                     __uint_as_float(acc[cb * 32 + i + 2 * h + 1]) * inv);
                             w[h] = *reinterpret_cast<uint32_t *>(&v);
                         }
                         const int chunk = (cb % 2) * 4 + i / 8;
