@@ -82,6 +82,16 @@ def test_small_shapes_kl(dd, oracle_mod, B, P, K, V, flagged, mode):
             assert ref["out_mask"][fl].any() and not ref["out_mask"][fl].all()
 
 
+@pytest.mark.parametrize("P", [700, 1100])
+def test_long_sequences(dd, oracle_mod, P):
+    """Sequences longer than the register-resident decision stage holds (512 positions) and than
+    its staged form holds (1024): the fold kernel's deciding warp takes the general path."""
+    hidden, weight, tokens, flags = synth.lm_head_inputs(2, P, 64, 520, "uniform_25_100", seed=P)
+    compare(dd, oracle_mod, hidden, weight, tokens, flags, CONF | PROB, 0.05, 9, 11)
+    dh, dw, vh, vw, tokens, flags = synth.lm_head_pair_inputs(2, P, 64, 520, "uniform_25_100", 0.2, seed=P + 1)
+    compare(dd, oracle_mod, vh, vw, tokens, flags, KL, 0.5, 9, 11, drafter=(dh, dw))
+
+
 def test_kl_tells_the_two_models_apart(dd, oracle_mod):
     """The drafter's pair and the verifier's pair swapped: D_KL(p_V || p_D) is another number."""
     dh, dw, vh, vw, tokens, flags = synth.lm_head_pair_inputs(1, 64, 128, 2000, 64, 0.2, seed=5)
