@@ -135,6 +135,73 @@ __device__ __forceinline__ float weights_to_tmem(const float (&s)[kBlockN], int 
     return sum2.x + sum2.y;
 }
 
+// One key tile of one query row, shared by both attention kernels: reads the row's 128 scores
+// from tensor memory (the S product has completed), weights them against the reference point the
+// row inherits (the first tile of a row takes its own maximum) and writes P over S.  Only a row
+// whose maximum turns out to have grown past the reference point by more than the allowed step
+// moves it, rescales O in tensor memory (which holds the sum over the earlier tiles once the
+// barrier o_full_bar has completed the phase o_parity) and weights the tile again.  Returns 0, or
+// the error code of the wait that expired.  The caller hands P over (wait for the stores, fence,
+// arrive).
+template <int D>
+__device__ __forceinline__ unsigned softmax_tile(uint32_t tS, uint32_t tO, uint32_t o_full_bar, uint32_t o_parity,
+                                                 bool first, int valid, float c, float &m_ref, float &l_run)
+{
+    float s[kBlockN];
+#pragma unroll
+    for (int cb = 0; cb < kBlockN / 32; ++cb)
+        tmem_ld32(tS + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cb * 32]));
+    tmem_wait_ld();
+    const bool masked = valid < kBlockN;
+    if (first) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
+    float mx;
+    float sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
+                       : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
+    const bool move = mx * c > m_ref + kRescaleStep;
+    if (__any_sync(0xffffffffu, move)) {
+        const float m_new = move ? mx * c : m_ref;
+        const float alpha = ex2(m_ref - m_new);       // 1 where the row does not move
+        m_ref = m_new;
+        l_run *= alpha;
+        if (!mbar_wait(o_full_bar, o_parity)) return kErrWaitO;
+        tc_fence_after();
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+            uint32_t r[32];
+            tmem_ld32(tO + cb * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st32(tO + cb * 32, r);
+        }
+        tmem_wait_st();                               // the first weights are overwritten next
+        sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
+                     : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
+    }
+    l_run += sum;
+    return 0;
+}
+
+// 32 columns of one output row, scaled, rounded to bf16 and written to the staging tile in the
+// 128-byte-swizzled layout of the output tensor map (`stage` = the row's first byte in the tile,
+// r = the row, cb = which 32 columns).
+__device__ __forceinline__ void columns_to_staging(const uint32_t *acc, float f, uint32_t stage, int r, int cb)
+{
+    constexpr uint32_t kBoxBytes = 128 * 128;
+    const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * f, __uint_as_float(acc[i + 2 * h + 1]) * f);
+            w[h] = *reinterpret_cast<uint32_t *>(&v);
+        }
+        const int chunk = (cb % 2) * 4 + i / 8;          // 16-byte chunk of the 128-byte row
+        st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
+    }
+}
+
 // kBlock = false: the square, head-major, unpadded case of dd_bidir_attention with nothing of the
 // general case compiled in.
 template <int D, bool kBlock>
@@ -247,45 +314,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const int j = j_first + i * j_step;
                 if (!mbar_wait(bar_s_full(g), i & 1)) { err = kErrWaitS; break; }
                 tc_fence_after();
-                float s[kBlockN];
-#pragma unroll
-                for (int cb = 0; cb < kBlockN / 32; ++cb)
-                    tmem_ld32(tS + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cb * 32]));
-                tmem_wait_ld();
-
                 const int valid = keys - j * kBlockN;      // keys of this tile that exist
                 const bool masked = valid < kBlockN;
-                // The first tile takes its reference point from its own maximum.  Later tiles are
-                // weighted against the reference point they inherit, in one pass, and only a row
-                // whose maximum turns out to have grown past it by more than the allowed step moves
-                // the reference point, rescales O and weights the tile again.
-                if (i == 0) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
-                float mx;
-                float sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
-                                   : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
-                const bool move = mx * c > m_ref + kRescaleStep;
-                if (__any_sync(0xffffffffu, move)) {
-                    const float m_new = move ? mx * c : m_ref;
-                    const float alpha = ex2(m_ref - m_new);       // 1 where the row does not move
-                    m_ref = m_new;
-                    l_run *= alpha;
-                    // O_g holds the sum over tiles < j once the previous P V has completed
-                    if (!mbar_wait(bar_o_full(g), (i - 1) & 1)) { err = kErrWaitO; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int cb = 0; cb < D / 32; ++cb) {
-                        uint32_t r[32];
-                        tmem_ld32(tO + cb * 32, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st32(tO + cb * 32, r);
-                    }
-                    tmem_wait_st();                               // the first weights are overwritten next
-                    sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
-                                 : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
-                }
-                l_run += sum;
+                // O_g holds the sum over tiles < j once the previous P V has completed
+                err = softmax_tile<D>(tS, tO, bar_o_full(g), (uint32_t)(i - 1) & 1, i == 0, valid, c, m_ref, l_run);
+                if (err) break;
                 if (kBlock && masked) {
                     // Keys past the end of the sequence have weight zero, but 0 x NaN is NaN in the
                     // product P V, and padding may hold any bit pattern: clear their value rows in
@@ -351,21 +384,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                         tmem_ld32(tO + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[cb * 32]));
                     tmem_wait_ld();
 #pragma unroll
-                    for (int cb = 0; cb < D / 32; ++cb) {
-                        const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
-#pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[cb * 32 + i + 2 * h]) * inv,
-                                                                         __uint_as_float(acc[cb * 32 + i + 2 * h + 1]) * inv);
-                                w[h] = *reinterpret_cast<uint32_t *>(&v);
-                            }
-                            const int chunk = (cb % 2) * 4 + i / 8;         // 16-byte chunk of the 128-byte row
-                            st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
-                        }
-                    }
+                    for (int cb = 0; cb < D / 32; ++cb) columns_to_staging(&acc[cb * 32], inv, stage, r, cb);
                 } else
 #pragma unroll
                 for (int cb = 0; cb < D / 32; ++cb) {
@@ -385,20 +404,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
                         for (int i = 0; i < 32; ++i) acc[i] = 0u;       // no key: nothing was accumulated
                     }
-                    const uint32_t box = stage + (cb / 2) * kBoxBytes;   // 64 columns per box
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const float f = (kBlock && split) ? 1.f : inv;      // split: already weighted
-                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[i + 2 * h]) * f,
-                                                                     __uint_as_float(acc[i + 2 * h + 1]) * f);
-                            w[h] = *reinterpret_cast<uint32_t *>(&v);
-                        }
-                        const int chunk = (cb % 2) * 4 + i / 8;         // 16-byte chunk of the 128-byte row
-                        st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
-                    }
+                    columns_to_staging(acc, (kBlock && split) ? 1.f : inv, stage, r, cb);      // split: already weighted
                 }
                 fence_proxy_async_smem();
             }

@@ -110,40 +110,9 @@ attention_persistent_kernel(const __grid_constant__ CUtensorMap tm_q, const __gr
             for (int j = 0; j < nkv; ++j, ++t_run) {
                 if (!mbar_wait(bar_s_full(g), t_run & 1)) { err = kErrWaitS; break; }
                 tc_fence_after();
-                float s[kBlockN];
-#pragma unroll
-                for (int cb = 0; cb < kBlockN / 32; ++cb)
-                    tmem_ld32(tS + cb * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cb * 32]));
-                tmem_wait_ld();
-                const int valid = p.Nkv - j * kBlockN;
-                const bool masked = valid < kBlockN;
-                if (j == 0) m_ref = (masked ? row_max<true>(s, valid) : row_max<false>(s, valid)) * c;
-                float mx;
-                float sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
-                                   : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
-                const bool move = mx * c > m_ref + kRescaleStep;
-                if (__any_sync(0xffffffffu, move)) {
-                    const float m_new = move ? mx * c : m_ref;
-                    const float alpha = ex2(m_ref - m_new);
-                    m_ref = m_new;
-                    l_run *= alpha;
-                    // O_g holds the sum over this item's tiles < j once the previous P V has completed
-                    if (!mbar_wait(bar_o_full(g), (t_run - 1) & 1)) { err = kErrWaitO; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int cb = 0; cb < D / 32; ++cb) {
-                        uint32_t r[32];
-                        tmem_ld32(tO + cb * 32, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st32(tO + cb * 32, r);
-                    }
-                    tmem_wait_st();
-                    sum = masked ? weights_to_tmem<true>(s, valid, c, m_ref, tS, mx)
-                                 : weights_to_tmem<false>(s, valid, c, m_ref, tS, mx);
-                }
-                l_run += sum;
+                // O_g holds the sum over this item's tiles < j once the previous P V has completed
+                err = softmax_tile<D>(tS, tO, bar_o_full(g), (t_run - 1) & 1, j == 0, p.Nkv - j * kBlockN, c, m_ref, l_run);
+                if (err) break;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar_p_full(g));
@@ -173,21 +142,7 @@ attention_persistent_kernel(const __grid_constant__ CUtensorMap tm_q, const __gr
                 tc_fence_before();
                 mbar_arrive(bar_o_free(g));
 #pragma unroll
-                for (int cb = 0; cb < D / 32; ++cb) {
-                    const uint32_t box = stage + (cb / 2) * kBoxBytes;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(acc[cb * 32 + i + 2 * h]) * inv,
-                                                                     __uint_as_float(acc[cb * 32 + i + 2 * h + 1]) * inv);
-                            w[h] = *reinterpret_cast<uint32_t *>(&v);
-                        }
-                        const int chunk = (cb % 2) * 4 + i / 8;
-                        st_shared_v4(box + ((chunk ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
-                    }
-                }
+                for (int cb = 0; cb < D / 32; ++cb) columns_to_staging(&acc[cb * 32], inv, stage, r, cb);
                 fence_proxy_async_smem();
             }
             // every thread of the warpgroup comes here, also after an expired wait
