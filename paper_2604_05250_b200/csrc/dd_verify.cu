@@ -455,9 +455,9 @@ int make_matrix_tmap(CUtensorMap *m, const void *base, long n_rows, int K, int b
 // Vocabulary entries per work item: the multiple of 32 (at most `max_n`, at least half of it) for
 // which the slowest CTA of `ctas` finishes first.  A work item of n entries takes about
 // (fixed + n) units of time: the hidden-state tiles it loads and the MMAs' shared-memory reads of
-// them do not shrink with n.  Measured at K = 4096 (time per item against n): fixed = 54 for one
-// product per item, 157 for the KL mode's two.  Counting n alone picked tiles of 128 entries at 4096
-// rows, 25 % slower than 256.
+// them do not shrink with n.  Measured at K = 4096 (time per item against n, tile widths forced):
+// fixed = 140 for one product per item, 157 for the KL mode's two.  Counting n alone picked tiles
+// of 128 entries at 4096 rows, 25 % slower than 256.
 int pick_tile_n(int V, long row_blocks, int ctas, int max_n, int fixed)
 {
     int best = max_n;
@@ -498,7 +498,7 @@ extern "C" int dd_lm_head_verify(const void *drafter_hidden, const void *drafter
     ddlm::LmParams q;
     q.rows = (int)rows; q.K = K; q.V = V;
     q.row_blocks = (int)((rows + ddlm::kRowsPerItem - 1) / ddlm::kRowsPerItem);
-    q.N = kl ? pick_tile_n(V, q.row_blocks, sms, ddlm::kMaxN / 2, 157) : pick_tile_n(V, q.row_blocks, sms, ddlm::kMaxN, 54);
+    q.N = kl ? pick_tile_n(V, q.row_blocks, sms, ddlm::kMaxN / 2, 157) : pick_tile_n(V, q.row_blocks, sms, ddlm::kMaxN, 140);
     q.n_tiles = (V + q.N - 1) / q.N;
     if (rows * q.n_tiles >= (1L << 31) - (1L << 24)) return DD_ERR_UNSUPPORTED;
 
