@@ -223,8 +223,11 @@ int pick_pieces(int V, long rows, int sms, long max_partials, bool kl)
     int k = 4;
     const long want = 2L * kSConsumers * sms;
     while (k > 1 && rows * chunks_of(k) < want) k >>= 1;
-    // with many units per warp the coarsest cut costs least (cfg2 shape: 5.95 against 5.76 TB/s)
-    if (k == 4 && k_max == 8 && rows * chunks_of(8) >= 8 * want) k = 8;
+    // The coarsest cut costs least (half the chunk ends, half the partials to fold and to publish)
+    // as long as every CTA still gets about two units per streaming warp: cfg2 shape 5.95 against
+    // 5.76 TB/s, cfg1 35.0 against 36.8 us; below that the ranges no longer balance (512 rows of a
+    // 32000-entry vocabulary: 30.0 against 27.5 us).
+    if (k == 4 && k_max == 8 && rows * chunks_of(8) >= 24L * sms) k = 8;
     while (max_partials > 0 && k < k_max && rows * chunks_of(k) > max_partials) k <<= 1;
     return k;
 }
