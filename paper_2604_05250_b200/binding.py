@@ -40,11 +40,37 @@ def lib() -> ctypes.CDLL:
     """Loads libdualdiff.so (once).  Raises if it has not been built."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
+        _lib = load(LIB_PATH)
+    return _lib
+
+
+class use_library:
+    """Context manager: the wrappers below call the library at `path` (for instance the
+    bounds-checked build) instead of libdualdiff.so until the block ends."""
+
+    def __init__(self, path):
+        self.path = path
+
+    def __enter__(self):
+        global _lib
+        self.saved = _lib
+        _lib = load(self.path)
+        return _lib
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self.saved
+        return False
+
+
+def load(path) -> ctypes.CDLL:
+    """Loads one build of the library and declares its entry points."""
+    if True:
+        if not os.path.exists(path):
             raise RuntimeError(
-                f"{LIB_PATH} is missing: build it with `python -m paper_2604_05250_b200.build`; "
+                f"{path} is missing: build it with `python -m paper_2604_05250_b200.build`; "
                 "there is no fallback implementation")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         vp, i32, f32, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint64
         attn = [vp, vp, vp, vp, i32, i32, i32, i32, f32, vp]
         ver = [vp, vp, vp, vp, i32, f32, i32, u64, vp, vp, vp, i32, i32, i32, vp]
@@ -81,8 +107,7 @@ def lib() -> ctypes.CDLL:
         L.dd_status_string.restype = ctypes.c_char_p
         L.dd_last_cuda_error.argtypes = []
         L.dd_last_cuda_error.restype = ctypes.c_char_p
-        _lib = L
-    return _lib
+    return L
 
 
 def _check(status: int):

@@ -66,6 +66,10 @@ struct Smem {
     static constexpr int kNumBars = 2 + 2 * kStages + 6;
     static constexpr int kTmemSlot = kBars + 8 * kNumBars;
     static constexpr int kTotal = kTmemSlot + 16;
+    // every tile starts on the 1024-byte boundary the 128-byte swizzle needs, the barriers on 8 bytes,
+    // and the whole layout plus the alignment slack fits what one CTA may ask for
+    static_assert(kTileBytes % 1024 == 0 && kBars % 8 == 0, "tiles on swizzle boundaries, barriers on 8 bytes");
+    static_assert(kTotal + 1024 <= 227 * 1024, "shared memory of one CTA");
 };
 
 __device__ __forceinline__ void report(const AttnParams &p, unsigned code)

@@ -34,6 +34,8 @@ struct SmemP {
     static constexpr int kNumBars = 8 + 2 * kPStages + 8;
     static constexpr int kTmemSlot = kBars + 8 * kNumBars;
     static constexpr int kTotal = kTmemSlot + 16;
+    static_assert(kTileBytes % 1024 == 0 && kBars % 8 == 0, "tiles on swizzle boundaries, barriers on 8 bytes");
+    static_assert(kTotal + 1024 <= 227 * 1024, "shared memory of one CTA");
 };
 
 template <int D>

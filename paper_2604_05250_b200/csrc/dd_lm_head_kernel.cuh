@@ -65,7 +65,7 @@ struct LmParams {
 // last tile.  170 of 217 us on a 256-row, 143-tile problem were that CTA folding alone.)
 __device__ __forceinline__ void store_partial(const ddv::VerifyParams &p, const ddv::Partial &c, int row, int tile)
 {
-    ddv::Partial *dst = p.partials + (size_t)row * p.nchunks + tile;
+    ddv::Partial *dst = p.partials + ddv::checked(p, (long)row * p.nchunks + tile, (long)p.B * p.P * p.nchunks, ddv::kSitePartial);
     __stcg(reinterpret_cast<float4 *>(dst), make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d));
     __stcg(reinterpret_cast<float4 *>(dst) + 1, make_float4(c.s_d, c.t, 0.f, 0.f));
 }
@@ -78,7 +78,7 @@ __device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int
     int last = 0;
     if (lane == 0) {
         __threadfence();
-        last = atomicAdd(p.seq_counter + b, (unsigned)n) + (unsigned)n == (unsigned)p.P;
+        last = atomicAdd(p.seq_counter + ddv::checked(p, b, p.B, ddv::kSiteSeq), (unsigned)n) + (unsigned)n == (unsigned)p.P;
     }
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
     if (!last) return;
@@ -100,10 +100,12 @@ __global__ void __launch_bounds__(kFoldThreads) lm_head_fold_kernel(const ddv::V
         if (!p.flags[w]) return;
         float score;
         int argmax;
-        ddv::fold_partials<KL>(p.partials + (size_t)w * p.nchunks, p.nchunks, score, argmax);
+        ddv::fold_partials<KL>(p.partials + ddv::checked_run(p, (long)w * p.nchunks, p.nchunks, (long)rows * p.nchunks, ddv::kSitePartial),
+                               p.nchunks, score, argmax);
         if ((threadIdx.x & 31) == 0) {
-            __stcg(p.row_score + w, score);
-            __stcg(p.row_argmax + w, argmax);
+            const size_t row_at = ddv::checked(p, w, (long)p.B * p.P, ddv::kSiteRow);
+            __stcg(p.row_score + row_at, score);
+            __stcg(p.row_argmax + row_at, argmax);
         }
         __syncwarp();
         rows_done(p, w / p.P, 1);

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
     __shared__ DecideStage s_decide;                // decision stage (warp 0 only)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int row = blockIdx.x / p.nchunks;
+    const int row = (int)checked(p, blockIdx.x / p.nchunks, (long)p.B * p.P, kSiteFlag);
     const int chunk = blockIdx.x - row * p.nchunks;
 
     if (!p.flags[row]) {
@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const V
     }
     const int e_begin = chunk * p.chunk;
     const int n = min(p.chunk, p.V - e_begin);
-    const size_t off = (size_t)row * p.V + e_begin;
+    const size_t off = checked_run(p, (long)row * p.V + e_begin, n, (long)p.B * p.P * p.V, kSiteLogit);
 
     uint4 rv[kVecPerThread], rd[kVecPerThread];
     load_chunk_elementwise(p.verifier + off, n, tid, rv);

@@ -61,6 +61,37 @@ __device__ __forceinline__ void report_expired(const VerifyParams &p, unsigned c
     }
 }
 
+// Bounds-checked build (-DDD_BOUNDS_CHECK, `python -m paper_2604_05250_b200.build --check`): every
+// index these kernels form into a caller's tensor or into the library's scratch goes through
+// checked(), which compares it with the extent, records kErrBounds | site << 8 in the health word
+// and substitutes index 0 (a legal one) on a violation, so that the launch finishes and the host
+// reads the word.  In the normal build checked() is the identity.  (The attention kernels address
+// global memory through tensor maps only, which the hardware clips.)
+constexpr unsigned kErrBounds = 0xB000;
+enum : unsigned { kSitePartial = 1, kSiteRow = 2, kSiteSeq = 3, kSiteLogit = 4, kSiteOut = 5, kSiteFlag = 6 };
+#ifdef DD_BOUNDS_CHECK
+constexpr bool kBoundsChecked = true;
+#else
+constexpr bool kBoundsChecked = false;
+#endif
+__device__ __forceinline__ size_t checked(const VerifyParams &p, long index, long extent, unsigned site)
+{
+    if (kBoundsChecked && (index < 0 || index >= extent)) {
+        report_expired(p, kErrBounds | (site << 8));
+        return 0;
+    }
+    return (size_t)index;
+}
+// the last element of a run of n starting at index (n >= 1) is checked as well
+__device__ __forceinline__ size_t checked_run(const VerifyParams &p, long index, long n, long extent, unsigned site)
+{
+    if (kBoundsChecked && (index < 0 || n < 1 || index + n > extent)) {
+        report_expired(p, kErrBounds | (site << 8));
+        return 0;
+    }
+    return (size_t)index;
+}
+
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;

@@ -44,7 +44,8 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
 
     const int lane = threadIdx.x & 31;
     const unsigned full = 0xFFFFFFFFu;
-    const long base = (long)b * p.P;
+    // every access below is at base + i with i < P: one check of the sequence index covers them
+    const long base = (long)checked(params, b, params.B, kSiteSeq) * p.P;
     const bool kl_mode = p.algo == DD_MODE_KL;
     const int nk = (p.P + 31) / 32;                 // positions per lane (upper bound)
     const bool staged = stage != nullptr && p.P <= kDecideKeys;      // without a staging area: re-read from memory
@@ -245,7 +246,7 @@ __device__ __forceinline__ void row_done(const VerifyParams &p, int b, DecideSta
     int last = 0;
     if (lane == 0) {
         __threadfence();
-        last = atomicAdd(p.seq_counter + b, 1u) == (unsigned)(p.P - 1);
+        last = atomicAdd(p.seq_counter + checked(p, b, p.B, kSiteSeq), 1u) == (unsigned)(p.P - 1);
     }
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
     if (!last) return;
@@ -330,11 +331,14 @@ __device__ __forceinline__ void fold_row(const VerifyParams &p, int row, DecideS
     __threadfence();
     float score;
     int argmax;
-    fold_partials<KL>(p.partials + (size_t)row * p.nchunks, p.nchunks, score, argmax);
+    const long n_rows = (long)p.B * p.P;
+    fold_partials<KL>(p.partials + checked_run(p, (long)row * p.nchunks, p.nchunks, n_rows * p.nchunks, kSitePartial),
+                      p.nchunks, score, argmax);
     if (lane == 0) {
-        __stcg(p.row_score + row, score);
-        __stcg(p.row_argmax + row, argmax);
-        p.row_counter[row] = 0u;      // ready for the next launch
+        const size_t row_at = checked(p, row, n_rows, kSiteRow);
+        __stcg(p.row_score + row_at, score);
+        __stcg(p.row_argmax + row_at, argmax);
+        p.row_counter[row_at] = 0u;      // ready for the next launch
     }
     __syncwarp();
     row_done(p, row / p.P, stage);
@@ -352,7 +356,7 @@ __device__ __forceinline__ void publish_batch(const VerifyParams &p, const Parti
     const int row = __float_as_int(c.pad0), chunk = __float_as_int(c.pad1);
     const bool mine = lane < n;
     if (mine && chunk >= 0) {
-        Partial *dst = p.partials + (size_t)row * p.nchunks + chunk;
+        Partial *dst = p.partials + checked(p, (long)row * p.nchunks + chunk, (long)p.B * p.P * p.nchunks, kSitePartial);
         const float4 a = make_float4(c.m_v, c.s_v, __int_as_float(c.idx), c.m_d);
         const float4 bq = make_float4(c.s_d, c.t, 0.f, 0.f);
         __stcg(reinterpret_cast<float4 *>(dst), a);
@@ -360,7 +364,8 @@ __device__ __forceinline__ void publish_batch(const VerifyParams &p, const Parti
     }
     __threadfence();
     bool last = false;
-    if (mine && chunk >= 0) last = atomicAdd(p.row_counter + row, 1u) == (unsigned)(p.nchunks - 1);
+    if (mine && chunk >= 0)
+        last = atomicAdd(p.row_counter + checked(p, row, (long)p.B * p.P, kSiteRow), 1u) == (unsigned)(p.nchunks - 1);
     unsigned todo = __ballot_sync(full, last);
     while (todo) {
         const int src = __ffs(todo) - 1;

@@ -24,7 +24,8 @@ __device__ __noinline__ void decide_sequence_small(const VerifyParams params, in
     const float tau = params.tau;
     const uint32_t seed_lo = params.seed_lo, seed_hi = params.seed_hi;
     const bool kl_mode = algo == DD_MODE_KL;
-    const long base = (long)b * P;
+    // every access below is at base + i with i < P: one check of the sequence index covers them
+    const long base = (long)checked(params, b, params.B, kSiteSeq) * P;
 
     // lane l owns positions l, l + 32, ...: key (order-preserving image of the reliability, 0
     // outside the set), token and verifier argmax

@@ -31,7 +31,7 @@ __device__ __forceinline__ void pending_flush(const VerifyParams &p, Pending &pe
     if (pend.used == 0) return;
     __threadfence();
     unsigned int before = 0u;
-    if (pend.b >= 0) before = atomicAdd(p.seq_counter + pend.b, (unsigned)pend.cnt);
+    if (pend.b >= 0) before = atomicAdd(p.seq_counter + checked(p, pend.b, p.B, kSiteSeq), (unsigned)pend.cnt);
     for (int e = 0; e < pend.used; ++e) {
         const int b = __shfl_sync(full, pend.b, e);
         const unsigned after = __shfl_sync(full, before, e) + (unsigned)__shfl_sync(full, pend.cnt, e);
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 s_meta[warp][stage] = make_int4(fl, i_where, i_row, i_chunk);
                 const uint32_t bytes = (uint32_t)n * 2u;
                 const uint32_t dst = ring + stage * kSStageBytes;
-                const size_t off = (size_t)i_row * p.V + e_begin;
+                const size_t off = checked_run(p, (long)i_row * p.V + e_begin, n, n_rows * p.V, kSiteLogit);
                 sbar_expect_tx(bar, KL ? 2u * bytes : bytes);
                 bulk_load(dst, p.verifier + off, bytes, bar, policy);
                 if (KL) bulk_load(dst + kSStageBytes / 2, p.drafter + off, bytes, bar, policy);
@@ -293,8 +293,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 lane_reset(L);
                 if (!(isfinite(part.s_v) && isfinite(part.s_d) && isfinite(part.t) && part.m_v > -INFINITY)) {
                     const int begin = meta.w * p.chunk;
-                    part = careful_chunk_partial<KL>(p.verifier + (size_t)meta.z * p.V,
-                                                     KL ? p.drafter + (size_t)meta.z * p.V : nullptr,
+                    const size_t row_off = checked_run(p, (long)meta.z * p.V, p.V, n_rows * p.V, kSiteLogit);
+                    part = careful_chunk_partial<KL>(p.verifier + row_off, KL ? p.drafter + row_off : nullptr,
                                                      begin, min(p.V, begin + p.chunk));
                 }
                 const int slot = meta.y & 0xFFFF, local_row = meta.y >> 16;
@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                     const int from = __ffs(m) - 1;
                     const int row = __shfl_sync(full, e.row, from), slot0 = __shfl_sync(full, e.first_slot, from);
                     const int chunk0 = __shfl_sync(full, e.first_chunk, from), cnt = __shfl_sync(full, e.count, from);
-                    Partial *dst = p.partials + (size_t)row * nch + chunk0;
+                    Partial *dst = p.partials + checked_run(p, (long)row * nch + chunk0, cnt, n_rows * nch, kSitePartial);
                     for (int i = lane; i < 2 * cnt; i += 32)
                         __stcg(reinterpret_cast<float4 *>(dst) + i, reinterpret_cast<const float4 *>(s_table + slot0)[i]);
                 }
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                     __threadfence();
                     bool complete = false;
                     if (mine_ok && !e.whole)
-                        complete = atomicAdd(p.row_counter + e.row, (unsigned)e.count) + (unsigned)e.count == (unsigned)nch;
+                        complete = atomicAdd(p.row_counter + checked(p, e.row, n_rows, kSiteRow), (unsigned)e.count) + (unsigned)e.count == (unsigned)nch;
                     const unsigned fold = __ballot_sync(full, complete);
                     if (fold) __threadfence();
                     for (unsigned m = fold; m; m &= m - 1) {
@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                         const int row = __shfl_sync(full, e.row, from);
                         float score;
                         int argmax;
-                        fold_partials<KL>(p.partials + (size_t)row * nch, nch, score, argmax);
+                        fold_partials<KL>(p.partials + checked_run(p, (long)row * nch, nch, n_rows * nch, kSitePartial), nch, score, argmax);
                         if (lane == from) {
                             e.whole = 1;
                             e.score = score;
@@ -419,8 +419,9 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 // finished rows: store, and count them per sequence
                 const bool finished = mine_ok && e.whole;
                 if (finished) {
-                    __stcg(p.row_score + e.row, e.score);
-                    __stcg(p.row_argmax + e.row, e.argmax);
+                    const size_t row_at = checked(p, e.row, n_rows, kSiteRow);
+                    __stcg(p.row_score + row_at, e.score);
+                    __stcg(p.row_argmax + row_at, e.argmax);
                 }
                 unsigned fin = __ballot_sync(full, finished);
                 while (fin) {
