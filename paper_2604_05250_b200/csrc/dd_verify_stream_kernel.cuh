@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     __shared__ __align__(16) EventQueue s_queue;
     __shared__ int s_scan[kSWarps];
     __shared__ int s_abort;                                       // a bounded wait expired somewhere in the CTA
+    __shared__ int s_setup;                                       // 1: the flag scan is complete, 2: the first range is set up
     __shared__ DecideStage s_decide;                              // decision stage (publishing warp only)
 
     const unsigned full = 0xFFFFFFFFu;
@@ -87,8 +88,21 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
 
     // ---- every thread counts the flagged rows of its contiguous slice of the B*P rows; the block
     // scan gives each thread the number of flagged rows before its slice, and the total
+    // The publishing warp takes no part in the scan or in the set-up of the CTA's first range: it
+    // spends that time (and the first microseconds of streaming) on the rehearsal below, and learns
+    // through s_setup how far the streaming warps have come.
+    constexpr int kScanThreads = kSConsumers * 32;
+    const bool publisher = warp == kSPublisherWarp;
+    volatile int *setup_flag = &s_setup;
+    volatile int *abort_flag = &s_abort;
     const long n_rows = (long)p.B * p.P;
-    if (warp == kSPublisherWarp && lane < kSConsumers) {
+    if (publisher) {
+        if (lane == 0) *setup_flag = 0;
+        __threadfence_block();
+        __syncwarp();
+        cta_bar_arrive(1, kSThreads);         // the streaming warps pass this barrier after the flag is zero
+    }
+    if (publisher && lane < kSConsumers) {
         // Before anything is known about the flags: ask the L2 (and with it the address translation)
         // for the first lines this CTA would stream if every row were flagged, one unit per
         // streaming warp.  The first copies of a launch otherwise arrive up to 4 us apart, and a
@@ -112,12 +126,14 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             }
         }
     }
-    const long slice = (n_rows + kSThreads - 1) / kSThreads;
-    const long my_begin = min(n_rows, (long)tid * slice), my_end = min(n_rows, my_begin + slice);
-    int my_count = 0;
-    for (long r = my_begin; r < my_end; ++r) my_count += p.flags[r] != 0;
-    long my_prefix, total_flagged;
-    {
+    const long slice = (n_rows + kScanThreads - 1) / kScanThreads;
+    const long my_begin = publisher ? n_rows : min(n_rows, (long)tid * slice);
+    const long my_end = publisher ? n_rows : min(n_rows, my_begin + slice);
+    long my_prefix = 0, total_flagged = 0;
+    bool setup_lost = false;          // publishing warp: the streaming warps never reported
+    if (!publisher) {
+        int my_count = 0;
+        for (long r = my_begin; r < my_end; ++r) my_count += p.flags[r] != 0;
         int incl = my_count;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -128,15 +144,54 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         if (tid < kSConsumers * kSStages) sbar_init(s_addr(&s_full[0][0] + tid), 1);
         if (tid == 0) s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        __syncthreads();
+        cta_bar_sync(1, kSThreads);
         int before = 0, all = 0;
-        for (int w = 0; w < kSWarps; ++w) {
+        for (int w = 0; w < kSConsumers; ++w) {
             const int v = s_scan[w];
             if (w < warp) before += v;
             all += v;
         }
         my_prefix = (long)before + incl - my_count;
         total_flagged = all;
+        if (tid == 0) {
+            __threadfence_block();
+            *setup_flag = 1;
+        }
+    } else {
+        // nothing is finished yet: bring the code of the row fold and of the decision stage into the
+        // instruction caches now, not at the end of the launch, and decide the sequences without a
+        // single flagged row (this CTA's share of them)
+        __shared__ float s_rehearsal[2];
+        float sc;
+        int am;
+        Partial *fake = reinterpret_cast<Partial *>(s_decide.key);      // free until a sequence ends
+        {
+            Partial f;
+            f.m_v = 1.f + lane; f.s_v = 1.5f; f.idx = lane; f.m_d = 0.5f * lane; f.s_d = 1.25f; f.t = 0.125f;
+            f.pad0 = f.pad1 = 0.f;
+            fake[lane] = f;
+        }
+        __syncwarp();
+        fold_partials<KL>(fake, 32, sc, am);
+        if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
+        decide_sequence_rehearsal(p, &s_decide);
+        for (int b = blockIdx.x; b < p.B; b += gridDim.x)
+            if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
+        // the scan's result
+        int seen = 0;
+        for (unsigned spin = 0; spin < (1u << 22); ++spin) {
+            seen = __shfl_sync(full, *setup_flag, 0);             // the same answer in every lane
+            if (seen >= 1) break;
+            __nanosleep(64);
+        }
+        __threadfence_block();
+        if (seen >= 1) {
+            int all = 0;
+            for (int w = 0; w < kSConsumers; ++w) all += s_scan[w];
+            total_flagged = all;
+        } else {
+            setup_lost = true;        // no range for this warp; reported below
+        }
     }
     // equal ranges, each small enough for the table, their number a multiple of the CTAs
     const unsigned total_units = (unsigned)(total_flagged * nch);          // fits 31 bits (checked by the host)
@@ -145,7 +200,6 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     const unsigned n_ranges = rounds * gridDim.x;
     const unsigned range_len = total_units / n_ranges, range_extra = total_units % n_ranges;
     auto range_begin = [&](unsigned r) { return r * range_len + min(r, range_extra); };
-    volatile int *abort_flag = &s_abort;
 
     unsigned it = 0;                  // streaming warp: stages taken (across ranges)
     Pending pend;
@@ -153,12 +207,11 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     pend.cnt = 0;
     pend.target = 0;
     pend.used = 0;
-    bool rehearsed = false;
-    // sequences without a single flagged row pass through; this CTA's share of them
-    auto pass_through = [&]() {
-        for (int b = blockIdx.x; b < p.B; b += gridDim.x)
-            if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
-    };
+    if (setup_lost && lane == 0) {
+        *abort_flag = 1;
+        report_expired(p, kErrWaitQueue);
+    }
+    bool first_range = true;
 
     for (unsigned range = blockIdx.x; range < n_ranges; range += gridDim.x) {
         const unsigned lo = range_begin(range), hi = range_begin(range + 1);
@@ -166,8 +219,24 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         const int n_units = (int)(hi - lo);
         const unsigned f_lo = lo / (unsigned)nch, f_hi = (hi - 1) / (unsigned)nch;   // flagged-row ordinals the range touches
 
-        if (range != blockIdx.x) __syncthreads();                 // the previous range is fully drained
-        {
+        if (first_range && publisher) {
+            // the streaming warps set the CTA's first range up among themselves
+            int seen = 0;
+            for (unsigned spin = 0; spin < (1u << 22); ++spin) {
+                seen = __shfl_sync(full, *setup_flag, 0);
+                if (seen >= 2) break;
+                __nanosleep(64);
+            }
+            __threadfence_block();
+            if (seen < 2) {
+                if (lane == 0) {
+                    *abort_flag = 1;
+                    report_expired(p, kErrWaitQueue);
+                }
+                break;                                            // this warp only: the others see the flag
+            }
+        } else {
+            if (!first_range) __syncthreads();                    // the previous range is fully drained
             long ord = my_prefix;
             for (long r = my_begin; r < my_end && ord <= (long)f_hi; ++r) {
                 if (p.flags[r]) {
@@ -175,11 +244,22 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                     ++ord;
                 }
             }
-            for (int i = tid; i < (int)(f_hi - f_lo + 1); i += kSThreads) s_rowcnt[i] = 0u;
+            const int helpers = first_range ? kScanThreads : kSThreads;       // tid < helpers here
+            for (int i = tid; i < (int)(f_hi - f_lo + 1); i += helpers) s_rowcnt[i] = 0u;
             if (tid < kSQueue) s_queue.ready[tid] = 0u;
             if (tid == 0) s_queue.tail = s_queue.head = s_queue.done = s_queue.next_unit = 0u;
+            if (first_range) {
+                // no wait can have expired yet
+                cta_bar_sync(2, kScanThreads);
+                if (tid == 0) {
+                    __threadfence_block();
+                    *setup_flag = 2;
+                }
+            } else if (__syncthreads_or(*abort_flag)) {
+                break;                                            // the same answer in every thread
+            }
         }
-        if (__syncthreads_or(*abort_flag)) break;                 // the same answer in every thread
+        first_range = false;
 
         if (warp < kSConsumers) {
             // ================================================================= streaming warps
@@ -334,26 +414,6 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
             }
         } else {
             // ================================================================= publishing warp
-            if (!rehearsed) {
-                // nothing is finished yet: bring the code of the row fold and of the decision stage
-                // into the instruction caches now, not at the end of the launch
-                rehearsed = true;
-                __shared__ float s_rehearsal[2];
-                float sc;
-                int am;
-                Partial *fake = reinterpret_cast<Partial *>(s_decide.key);      // free until a sequence ends
-                {
-                    Partial f;
-                    f.m_v = 1.f + lane; f.s_v = 1.5f; f.idx = lane; f.m_d = 0.5f * lane; f.s_d = 1.25f; f.t = 0.125f;
-                    f.pad0 = f.pad1 = 0.f;
-                    fake[lane] = f;
-                }
-                __syncwarp();
-                fold_partials<KL>(fake, 32, sc, am);
-                if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
-                decide_sequence_rehearsal(p, &s_decide);
-                pass_through();
-            }
             unsigned int head = 0;
             for (unsigned idle = 0;;) {
                 const unsigned int mine = head + lane;
@@ -435,7 +495,6 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         }
     }
 
-    if (warp == kSPublisherWarp && !rehearsed) pass_through();      // this CTA had no range
     __syncthreads();
     if (*abort_flag) {
         // a wait expired: give copies that may still be in flight time to land before the shared
