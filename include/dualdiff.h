@@ -63,7 +63,9 @@ enum {
  *     out[b,h,i,:] = sum_j softmax_j(scale * q[b,h,i,:] . k[b,h,j,:]) v[b,h,j,:],
  * j over all N positions.  q, k, v, out: [B,H,N,D] bf16, D innermost, 16-byte
  * aligned, out not overlapping the inputs.  Scores and the softmax are
- * accumulated in fp32; the result is rounded to bf16 once.
+ * accumulated in fp32 (weights relative to a per-row reference point that may lag the
+ * row maximum by a factor of up to 2^24: the result is finite for |v| * N < 2^100);
+ * the result is rounded to bf16 once.
  * Supported: D in {64,128}; any N >= 1; scale >= 0; B*H*ceil(N/128) < 2^31.
  * Errors: DD_ERR_INVALID_ARG (null pointer, B/H/N/D <= 0, scale not finite),
  * DD_ERR_UNSUPPORTED (other D, negative scale, misaligned pointer), DD_ERR_CUDA.

@@ -16,8 +16,9 @@
 // into one FMA), writes P = 2^(S - m) as bf16 over the first half of the S columns,
 // and O_g += P V is a second MMA whose A operand is read from tensor memory.  While
 // one tile's softmax runs, the tensor core works on the other tile.  The reference
-// point m of a row only moves when the row maximum has grown by more than 2^8
-// (P stays below 256, exact enough in bf16 and harmless in the fp32 sum); only then
+// point m of a row only moves when the row maximum has outgrown it by more than 2^24
+// (a power-of-two factor common to P and to the row sum changes neither bf16's nor
+// fp32's relative precision; the step only has to leave fp32 its range); only then
 // is O rescaled in tensor memory.  O is normalised by the row sum at the end and
 // rounded to bf16 once.
 #include <cuda.h>
@@ -41,7 +42,12 @@ constexpr int kThreads = 384;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kLoadWarp = 8, kMmaWarp = 9;
 constexpr uint32_t kTmemCols = 512; // S_0 [0,128)  S_1 [128,256)  O_0 [256,256+D)  O_1 [256+D,256+2D)
-constexpr float kRescaleStep = 8.f; // log2 of the largest P tolerated before the reference point moves
+// log2 of the largest P tolerated before the reference point moves.  A move costs the row's warp a
+// wait for the previous P V product, a pass over the accumulator in tensor memory and a second
+// weighting of the tile: with a step of 8, rows whose scores are peaked (a planted low-rank
+// component; trained heads) moved often enough to cost 25-40 % of the throughput.  With 24 the sum
+// of a row's weights stays below N * 2^24 and fp32 holds O for |v| * N < 2^100.
+constexpr float kRescaleStep = 24.f;
 
 enum : unsigned { kErrWaitQ = 0x100, kErrWaitKV = 0x200, kErrWaitS = 0x300, kErrWaitO = 0x400,
                   kErrWaitP = 0x500, kErrWaitSlot = 0x600 };

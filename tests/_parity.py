@@ -35,10 +35,25 @@ def attention_max_abs_bar(oracle_out):
     return ATTN_MAX_ABS * np.maximum(1.0, np.exp2(np.floor(np.log2(mag)) - 1.0))
 
 
-def check_attention(gpu_out_f64, oracle_out):
+# Stress inputs only (planted strength 6: one or two keys carry a row).  Where the exact value
+# lies in [2, 4), half a unit of the bf16 output is already 2^-7 = 7.8e-3, and the bf16 rounding
+# of the weights (2^-9 relative each) of two keys that share a row adds up to
+# 2^-8 |v1 - v2| / 4 = 3.9e-3 for |v1 - v2| = 4: 1.17e-2 together.  Such elements are rare
+# (they need both roundings near their worst case): at most STRESS_OVER_SHARE of all elements may
+# pass 1e-2, none may pass STRESS_MAX_ABS.
+STRESS_MAX_ABS = 1.2e-2
+STRESS_OVER_SHARE = 1e-5
+
+
+def check_attention(gpu_out_f64, oracle_out, stress=False):
     diff = np.abs(gpu_out_f64 - oracle_out)
     assert np.isfinite(gpu_out_f64).all()
-    over = diff > attention_max_abs_bar(oracle_out)
+    bar = attention_max_abs_bar(oracle_out)
+    if stress:
+        late = (diff > bar) & (np.abs(oracle_out) >= 2.0) & (np.abs(oracle_out) < 4.0)
+        assert late.sum() <= max(1, int(STRESS_OVER_SHARE * diff.size)), f"{late.sum()} of {diff.size} elements over 1e-2"
+        bar = np.where(late, STRESS_MAX_ABS, bar)
+    over = diff > bar
     assert not over.any(), (f"{over.sum()} elements over the max-abs bar; worst {diff[over].max():.3e} "
                             f"at |exact| = {np.abs(oracle_out)[over][diff[over].argmax()]:.3f}")
     assert diff.mean() <= ATTN_MEAN_ABS, f"mean-abs {diff.mean():.3e}"
