@@ -115,6 +115,21 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 }
 
 // Running state of one lane over the pieces of a chunk.
+// Packed bf16x2 maximum of two words.
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
+{
+    const __nv_bfloat162 m = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+    return *reinterpret_cast<const uint32_t *>(&m);
+}
+
+// A chunk whose sum T = sum e (l_D - l_V) exceeds this many times its sum of weights S_D cannot come
+// from logits of any model (an average difference of 10^4 nats); it is what a token excluded by
+// the verifier alone leaves behind once -inf has been raised to the lowest finite bf16
+// (3.4e38 times the token's weight).  Such a chunk goes to the scalar routine, which returns the
+// infinite divergence.  A token the drafter gives a probability below 10^4 / 3.4e38 = 3e-35
+// of the chunk's mass escapes the test and counts as excluded by both models.
+constexpr float kExcludedExcess = 1e4f;
+
 struct LaneState {
     uint32_t max2_v;           // packed bf16x2 running maxima of the verifier (even / odd logits of the lane's words)
     uint32_t where2_v;         // per half: ordinal of the word that first attained that maximum
@@ -198,10 +213,19 @@ __device__ __forceinline__ void lane_pass2(LaneState &L, const uint4 (&rv)[kVecP
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
         if (kFull || (lane + j * 32) * 8 < n) {
-            const uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
-            const uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
+            uint32_t wv[4] = {rv[j].x, rv[j].y, rv[j].z, rv[j].w};
+            uint32_t wd[4] = {rd[j].x, rd[j].y, rd[j].z, rd[j].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
+                if (KL) {
+                    // An excluded token (logit -inf) has weight 2^(-inf) = 0 either way, but in
+                    // e * (d - v) it would be 0 * inf: both logits are raised to the lowest finite
+                    // bf16 first, so the term of a token the drafter excludes is an exact 0
+                    // whatever the verifier says.  (A token only the verifier excludes then adds
+                    // e * 3.4e38 instead of infinity: kExcludedExcess below catches that.)
+                    wv[h] = bf16x2_max(wv[h], 0xFF7FFF7Fu);
+                    wd[h] = bf16x2_max(wd[h], 0xFF7FFF7Fu);
+                }
                 const float2 v2 = make_float2(bf16lo(wv[h]), bf16hi(wv[h]));
                 const float2 a = __ffma2_rn(v2, log2e2, nMv2);
                 s_v = __fadd2_rn(s_v, make_float2(ex2_approx(a.x), ex2_approx(a.y)));

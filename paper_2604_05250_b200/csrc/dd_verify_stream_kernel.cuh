@@ -371,7 +371,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                 // of a row hands the row on
                 Partial part = lanes_to_partial<KL>(L, meta.w * p.chunk, lane);
                 lane_reset(L);
-                if (!(isfinite(part.s_v) && isfinite(part.s_d) && isfinite(part.t) && part.m_v > -INFINITY)) {
+                if (!(isfinite(part.s_v) && isfinite(part.s_d) && isfinite(part.t) && part.m_v > -INFINITY) ||
+                    (KL && fabsf(part.t) > kExcludedExcess * part.s_d)) {
                     const int begin = meta.w * p.chunk;
                     const size_t row_off = checked_run(p, (long)meta.z * p.V, p.V, n_rows * p.V, kSiteLogit);
                     part = careful_chunk_partial<KL>(p.verifier + row_off, KL ? p.drafter + row_off : nullptr,

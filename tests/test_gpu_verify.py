@@ -249,6 +249,26 @@ def test_results_do_not_depend_on_the_grid(dd, oracle_mod, cta_cap):
         check_verify(*ref, oracle_mod.verify(d_in, ver, tokens, flags, mode, tau, k, seed), flags, tokens)
 
 
+@pytest.mark.parametrize("V", [20000, 1003])
+def test_token_excluded_by_the_verifier_alone(dd, oracle_mod, V):
+    """p_V(x) = 0 where p_D(x) > 0: the divergence of Eq. 5 is infinite, in the oracle and in both
+    kernels (the streaming path meets the token as a finite logit of -3.4e38 and must notice)."""
+    ninf = np.uint16(0xFF80)
+    dra, ver, tokens, flags = synth.verify_inputs(2, 12, V, 12, 0.25, seed=77 + V)
+    rng = np.random.default_rng(V + 1)
+    ver[0, 2, rng.choice(V, size=5, replace=False)] = ninf            # five ordinary tokens
+    top = int(np.argmax(synth.bf16_bits_to_f32(dra[1, 3])))
+    ver[1, 3, top] = ninf                                              # the drafter's most likely token
+    both = rng.choice(V, size=40, replace=False)
+    dra[1, 4, both] = ninf; ver[1, 4, both] = ninf                     # a row that stays finite
+    tokens[:] = np.argmax(synth.bf16_bits_to_f32(dra), axis=2)
+    _, ref, got = compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 3, 7)
+    inf_at = np.zeros((2, 12), dtype=bool)
+    inf_at[0, 2] = inf_at[1, 3] = True
+    assert np.isposinf(ref["out_score"][inf_at]).all() and np.isposinf(got[2][inf_at]).all()
+    assert np.isfinite(ref["out_score"][~inf_at]).all() and np.isfinite(got[2][~inf_at]).all()
+
+
 @pytest.mark.parametrize("V", [4096, 20000, 1003])
 def test_excluded_tokens(dd, oracle_mod, V):
     """Logits of -inf (banned or padded vocabulary entries) at shared and at drafter-only
