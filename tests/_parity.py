@@ -65,10 +65,15 @@ def check_verify(gpu_tokens, gpu_mask, gpu_score, ref, flags, tokens_in, score_a
     flags = flags.astype(bool)
     exempt = ref["exempt"].astype(bool)
     o_score = ref["out_score"]
-    tol = np.maximum(SCORE_REL * np.abs(o_score), score_abs)
-    bad = np.abs(gpu_score.astype(np.float64) - o_score) > tol
-    assert not bad.any(), (f"{bad.sum()} scores out of tolerance; worst "
-                           f"{np.abs(gpu_score - o_score).max():.3e}")
+    g_score = gpu_score.astype(np.float64)
+    unbounded = np.isinf(o_score)                   # a token only the verifier excludes: KL = +inf
+    assert np.array_equal(unbounded, np.isinf(g_score)), "infinite scores at different positions"
+    assert (g_score[unbounded] == o_score[unbounded]).all()
+    fin = ~unbounded
+    tol = np.maximum(SCORE_REL * np.abs(o_score[fin]), score_abs)
+    err = np.abs(g_score[fin] - o_score[fin])
+    bad = ~(err <= tol)                             # a NaN is out of tolerance too
+    assert not bad.any(), f"{bad.sum()} scores out of tolerance; worst {np.nanmax(err):.3e}"
     strict = ~exempt
     mism_mask = (gpu_mask != ref["out_mask"]) & strict
     assert not mism_mask.any(), f"{mism_mask.sum()} remask decisions differ outside the exempt set"
