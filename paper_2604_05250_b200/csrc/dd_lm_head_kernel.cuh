@@ -72,7 +72,7 @@ __device__ __forceinline__ void store_partial(const ddv::VerifyParams &p, const 
 
 // n more rows of sequence b are accounted for (warp-level); the warp that accounts for the last
 // of the P rows decides the sequence.
-__device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int n)
+__device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int n, ddv::DecideStage *stage)
 {
     const int lane = threadIdx.x & 31;
     int last = 0;
@@ -84,7 +84,7 @@ __device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int
     if (!last) return;
     __threadfence();
     if (lane == 0) p.seq_counter[b] = 0u;      // ready for the next launch
-    ddv::decide_sequence(p, b, nullptr);
+    ddv::decide_sequence(p, b, stage);
 }
 
 // Second launch of dd_lm_head_verify: one warp per row folds the row's tile partials (fp64, tile
@@ -92,9 +92,14 @@ __device__ __forceinline__ void rows_done(const ddv::VerifyParams &p, int b, int
 // for the rows that are not flagged; the warp that accounts for a sequence's last row runs the
 // decision stage.  The partials were written by the previous kernel on the stream.
 constexpr int kFoldThreads = 128;
+constexpr int kFoldDecideKeys = 2048;      // keys of one sequence each warp can keep in shared memory
 template <bool KL>
 __global__ void __launch_bounds__(kFoldThreads) lm_head_fold_kernel(const ddv::VerifyParams p, int rows)
 {
+    __shared__ uint32_t s_keys[kFoldThreads / 32][kFoldDecideKeys];
+    ddv::DecideStage stage;
+    stage.key = s_keys[threadIdx.x >> 5];
+    stage.capacity = kFoldDecideKeys;
     const int w = blockIdx.x * (kFoldThreads / 32) + (threadIdx.x >> 5);     // rows first, then sequences
     if (w < rows) {
         if (!p.flags[w]) return;
@@ -108,12 +113,12 @@ __global__ void __launch_bounds__(kFoldThreads) lm_head_fold_kernel(const ddv::V
             __stcg(p.row_argmax + row_at, argmax);
         }
         __syncwarp();
-        rows_done(p, w / p.P, 1);
+        rows_done(p, w / p.P, 1, &stage);
     } else {
         const int b = w - rows;
         if (b >= p.B) return;
         const int unflagged = p.P - ddv::count_flagged(p, b);
-        if (unflagged > 0) rows_done(p, b, unflagged);
+        if (unflagged > 0) rows_done(p, b, unflagged, &stage);
     }
 }
 

@@ -145,11 +145,16 @@ __device__ __forceinline__ void warp_partial(const uint4 (&rv)[kVecPerThread], c
     out.pad0 = out.pad1 = 0.f;
 }
 
+constexpr int kEDecideKeys = 2048;      // keys of one sequence the element-wise kernel's deciding warp keeps in shared memory
+
 template <bool KL>
 __global__ void __launch_bounds__(kThreads, 3) verify_elementwise_kernel(const VerifyParams p)
 {
     __shared__ Partial warp_part[kWarps];
-    __shared__ DecideStage s_decide;                // decision stage (warp 0 only)
+    __shared__ uint32_t s_decide_keys[kEDecideKeys];   // decision stage (warp 0 only)
+    DecideStage s_decide;
+    s_decide.key = s_decide_keys;
+    s_decide.capacity = kEDecideKeys;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = (int)checked(p, blockIdx.x / p.nchunks, (long)p.B * p.P, kSiteFlag);

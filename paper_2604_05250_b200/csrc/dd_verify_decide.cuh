@@ -12,21 +12,26 @@ namespace ddv {
 // the score; positions above t are kept, and those equal to t are kept lowest index first
 // until k are kept in all.  This equals ranking by (reliability descending, index ascending).
 //
-// Lane l owns positions l, l+32, l+64, ...  The keys of a sequence of up to kDecideKeys
-// positions, with their tokens and argmaxes, are staged in the caller's shared memory; longer sequences re-read
-// them from memory on every pass.  The code runs once per sequence, from a cold instruction
-// cache: it is written as short loops, not unrolled.
+// Lane l owns positions l, l+32, l+64, ...  The keys of a sequence that fits the caller's staging
+// area are kept there (shared memory), and in registers as well while there are at most 32 per
+// lane; longer sequences re-read them from memory on every pass (33 passes of dependent loads:
+// two orders of magnitude slower, so callers size the area for the sequences they expect).
+// The code runs once per sequence, from a cold instruction cache: it is written as short loops,
+// not unrolled.
 // The parameters come by value: only this rare call copies them to the stack.  dry: every
 // load and every step, but no store.
-constexpr int kDecideKeys = 1024;
+constexpr int kDecideRegKeys = 1024;     // keys a warp can also hold in registers
 
-struct __align__(16) DecideStage {      // one per deciding warp, in shared memory
-    uint32_t key[kDecideKeys];
-    int32_t tok[kDecideKeys];      // tokens[b, i]
-    int32_t top[kDecideKeys];      // verifier argmax of position i
+// `dry` of the decision functions: 0 decides; a rehearsal makes every load and every step but no
+// store, and the short one walks through only two steps of the threshold search.
+constexpr int kDryFull = 1, kDryShort = 2;
+
+struct DecideStage {            // one per deciding warp
+    uint32_t *key;              // shared memory for `capacity` keys (at least 256: the rehearsal's table)
+    int capacity;
 };
 
-__device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int b, DecideStage *stage, bool dry)
+__device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int b, DecideStage *stage, int dry)
 {
     // Every field goes into a register once: the stores below are through generic pointers, after
     // which the compiler would have to read the by-value structure again.
@@ -48,7 +53,9 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
     const long base = (long)checked(params, b, params.B, kSiteSeq) * p.P;
     const bool kl_mode = p.algo == DD_MODE_KL;
     const int nk = (p.P + 31) / 32;                 // positions per lane (upper bound)
-    const bool staged = stage != nullptr && p.P <= kDecideKeys;      // without a staging area: re-read from memory
+    const bool staged = stage != nullptr && p.P <= stage->capacity;      // without a staging area: re-read from memory
+    uint32_t *const skey = staged ? stage->key : nullptr;
+    const bool in_regs = staged && p.P <= kDecideRegKeys;
 
     // key of position i: order-preserving image of its reliability, 0 outside the set.
     // Both loads are unconditional (the score slot exists for every position), so a pass
@@ -64,37 +71,31 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
         // they overlap), then the stores
         for (int r0 = 0; r0 < nk; r0 += 8) {
             uint32_t k[8];
-            int32_t tk[8], tp[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) k[u] = load_key(lane + 32 * (r0 + u));
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int i = lane + 32 * (r0 + u);
-                const int ic = min(i, p.P - 1);
-                k[u] = load_key(i);
-                tk[u] = p.tokens[base + ic];
-                tp[u] = __ldcg(p.row_argmax + base + ic);
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = lane + 32 * (r0 + u);
-                if (i < kDecideKeys) { stage->key[i] = k[u]; stage->tok[i] = tk[u]; stage->top[i] = tp[u]; }
+                if (r0 + u < nk) skey[i] = k[u];      // i < 32 nk <= capacity rounded up to 32 (the area is a multiple of 32)
             }
         }
         __syncwarp();
     }
-    auto key_at = [&](int r) -> uint32_t { return staged ? stage->key[lane + 32 * r] : load_key(lane + 32 * r); };
+    auto key_at = [&](int r) -> uint32_t { return staged ? skey[lane + 32 * r] : load_key(lane + 32 * r); };
     auto score_of = [&](uint32_t key) -> float {     // inverse of the key map (key != 0)
         const float rel = __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
         return kl_mode ? 0.0f - rel : rel;
     };
-    // number of keys of the whole sequence with key >= cand, or key > cand.  Staged keys are
-    // also held in registers (up to 32 per lane): the threshold search below makes 33 passes.
-    uint32_t kr[kDecideKeys / 32];
+    // number of keys of the whole sequence with key >= cand, or key > cand.  The threshold search
+    // below makes 33 passes: from registers (up to 32 keys per lane), else from the staging area,
+    // else from memory.
+    uint32_t kr[kDecideRegKeys / 32];
 #pragma unroll
-    for (int r = 0; r < kDecideKeys / 32; ++r) kr[r] = (staged && r < nk) ? stage->key[lane + 32 * r] : 0u;
+    for (int r = 0; r < kDecideRegKeys / 32; ++r) kr[r] = (in_regs && r < nk) ? skey[lane + 32 * r] : 0u;
     auto count_keys = [&](uint32_t cand, bool strictly) -> int {
         int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
-        if (staged) {
-            const uint32_t bound = strictly ? cand : cand - 1u;      // cand >= 1 when not strict
+        const uint32_t bound = strictly ? cand : cand - 1u;      // cand >= 1 when not strict
+        if (in_regs) {
             if (nk <= 8) {
 #pragma unroll
                 for (int r = 0; r < 8; r += 4) {
@@ -102,10 +103,23 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
                 }
             } else {
 #pragma unroll
-                for (int r = 0; r < kDecideKeys / 32; r += 4) {
+                for (int r = 0; r < kDecideRegKeys / 32; r += 4) {
                     c0 += kr[r] > bound; c1 += kr[r + 1] > bound; c2 += kr[r + 2] > bound; c3 += kr[r + 3] > bound;
                 }
             }
+        } else if (staged) {
+            // slots past the sequence hold 0 (the staging loop wrote load_key's 0 there)
+            // sixteen independent loads per step: a pass is bound by their issue, not their latency
+            const uint32_t *kp = skey + lane;
+            int r = 0;
+            for (; r + 15 < nk; r += 16) {
+#pragma unroll
+                for (int u = 0; u < 16; u += 4) {
+                    c0 += kp[32 * (r + u)] > bound; c1 += kp[32 * (r + u + 1)] > bound;
+                    c2 += kp[32 * (r + u + 2)] > bound; c3 += kp[32 * (r + u + 3)] > bound;
+                }
+            }
+            for (; r < nk; ++r) c0 += kp[32 * r] > bound;
         } else {
 #pragma unroll 4
             for (int r = 0; r < nk; ++r) {
@@ -162,27 +176,22 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
         }
     }
 
-    // final pass, four positions per lane at a time: first every load of the group (they are
+    // final pass, eight positions per lane at a time: first every load of the group (they are
     // independent, so they overlap), then the decisions and the stores
     int equal_seen = 0;         // positions equal to thr at lower indices
-    for (int r0 = 0; r0 < nk; r0 += 4) {
-        uint32_t key[4];
-        int32_t tok[4], top[4];
+    for (int r0 = 0; r0 < nk; r0 += 8) {
+        uint32_t key[8];
+        int32_t tok[8], top[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const int i = lane + 32 * (r0 + u);
             const bool in = r0 + u < nk && i < p.P;
             key[u] = r0 + u < nk ? key_at(r0 + u) : 0u;
-            if (staged) {
-                tok[u] = in ? stage->tok[i] : 0;
-                top[u] = in ? stage->top[i] : 0;
-            } else {
-                tok[u] = in ? p.tokens[base + i] : 0;
-                top[u] = (in && key[u] != 0u) ? __ldcg(p.row_argmax + base + i) : 0;
-            }
+            tok[u] = in ? p.tokens[base + i] : 0;
+            top[u] = (in && key[u] != 0u) ? __ldcg(p.row_argmax + base + i) : 0;
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const int r = r0 + u;
             if (r >= nk) break;                     // uniform
             const int i = lane + 32 * r;
@@ -219,7 +228,7 @@ __device__ __noinline__ void decide_sequence_impl(const VerifyParams params, int
 namespace ddv {
 
 // Short sequences are decided from registers, longer ones from the staging area.
-__device__ __forceinline__ void decide_dispatch(const VerifyParams &p, int b, DecideStage *stage, bool dry)
+__device__ __forceinline__ void decide_dispatch(const VerifyParams &p, int b, DecideStage *stage, int dry)
 {
     if (p.P <= 256) decide_sequence_small<8>(p, b, dry);
     else if (p.P <= 512) decide_sequence_small<16>(p, b, dry);
@@ -228,15 +237,15 @@ __device__ __forceinline__ void decide_dispatch(const VerifyParams &p, int b, De
 
 __device__ __forceinline__ void decide_sequence(const VerifyParams &p, int b, DecideStage *stage)
 {
-    decide_dispatch(p, b, stage, false);
+    decide_dispatch(p, b, stage, 0);
 }
 
 // Runs the decision code on sequence 0 without storing anything.  The decision runs once per
 // sequence, at the very end of a launch that has streamed the instruction lines out of every
 // cache; a warp with nothing to do yet calls this to bring them back in.
-__device__ __forceinline__ void decide_sequence_rehearsal(const VerifyParams &p, DecideStage *stage)
+__device__ __forceinline__ void decide_sequence_rehearsal(const VerifyParams &p, DecideStage *stage, bool brief)
 {
-    decide_dispatch(p, 0, stage, true);
+    decide_dispatch(p, 0, stage, brief ? kDryShort : kDryFull);
 }
 
 // One sequence has one more completed row; the warp that completes the sequence decides it.

@@ -7,7 +7,7 @@
 namespace ddv {
 
 template <int R>
-__device__ __noinline__ void decide_sequence_small(const VerifyParams params, int b, bool dry)
+__device__ __noinline__ void decide_sequence_small(const VerifyParams params, int b, int dry)
 {
     const int lane = threadIdx.x & 31;
     const unsigned full = 0xFFFFFFFFu;
@@ -91,7 +91,9 @@ __device__ __noinline__ void decide_sequence_small(const VerifyParams params, in
             keep_all = true;
         } else {
             topk_active = true;
-            for (int bit = 31; bit >= 0; --bit) {
+            // (a short rehearsal walks through two of the 32 steps: each waits for the one before
+            // it, and the whole search is a third of this function's time)
+            for (int bit = 31; bit >= (dry == kDryShort ? 30 : 0); --bit) {
                 const uint32_t cand = thr | (1u << bit);
                 if (count_above(cand - 1u) >= k_keep) thr = cand;      // keys >= cand
             }

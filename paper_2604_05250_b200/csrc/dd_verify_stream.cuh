@@ -49,6 +49,7 @@ constexpr int kSThreads = kSWarps * 32;
 constexpr int kSStages = 2;                                   // ring slots per streaming warp (three gain nothing)
 constexpr int kSStageBytes = 4096;
 constexpr int kSRingBytes = kSConsumers * kSStages * kSStageBytes;
+constexpr int kSDecideKeys = 8192;                            // keys of one sequence the publishing warp can keep in shared memory
 constexpr int kSQueue = 64;                                   // finished-row queue slots
 constexpr int kSTable = 640;                                  // chunk partials a CTA keeps per range
 constexpr int kPiece = 32 * kVecPerThread * 8;                // 1024 logits per tensor per stage (KL)

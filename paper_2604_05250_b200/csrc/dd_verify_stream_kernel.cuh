@@ -72,14 +72,27 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
     extern __shared__ __align__(128) unsigned char s_ring[];     // [warp][stage][kSStageBytes]
     __shared__ __align__(8) unsigned long long s_full[kSConsumers][kSStages];    // mbarriers: the stage holds data
     __shared__ __align__(16) int4 s_meta[kSConsumers][kSStages];  // what the stage holds
-    __shared__ __align__(16) Partial s_table[kSTable];            // chunk partials of the current range
+    // chunk partials of the current range; between ranges (every streaming warp has finished, every
+    // row event has been taken) the same memory holds the keys of the sequence being decided
+    constexpr int kTableSlots = kSDecideKeys * 4 / (int)sizeof(Partial);
+    static_assert(kTableSlots >= kSTable, "the table fits the area");
+    __shared__ __align__(16) Partial s_table[kTableSlots];       // kSTable slots in use as a table
+    __shared__ __align__(16) Partial s_fake[32];                   // the rehearsal's partials
     __shared__ int s_rows[kSTable + 2];                           // flagged rows the range touches
     __shared__ unsigned int s_rowcnt[kSTable + 2];                // their chunks stored so far
     __shared__ __align__(16) EventQueue s_queue;
     __shared__ int s_scan[kSWarps];
     __shared__ int s_abort;                                       // a bounded wait expired somewhere in the CTA
     __shared__ int s_setup;                                       // 1: the flag scan is complete, 2: the first range is set up
-    __shared__ DecideStage s_decide;                              // decision stage (publishing warp only)
+    // Decision stage of the publishing warp at the end of a range.  Anywhere else (sequences
+    // without a flagged row at the kernel's start; a flush in the middle of a range, which only
+    // ranges over more than 32 sequences, hence short ones, ever need) the table is in use and the
+    // decision runs without a key area.
+    DecideStage s_decide, s_no_area;
+    s_decide.key = reinterpret_cast<uint32_t *>(s_table);
+    s_decide.capacity = kSDecideKeys;
+    s_no_area.key = nullptr;
+    s_no_area.capacity = 0;
 
     const unsigned full = 0xFFFFFFFFu;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -164,7 +177,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         __shared__ float s_rehearsal[2];
         float sc;
         int am;
-        Partial *fake = reinterpret_cast<Partial *>(s_decide.key);      // free until a sequence ends
+        Partial *fake = s_fake;
         {
             Partial f;
             f.m_v = 1.f + lane; f.s_v = 1.5f; f.idx = lane; f.m_d = 0.5f * lane; f.s_d = 1.25f; f.t = 0.125f;
@@ -174,9 +187,8 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         __syncwarp();
         fold_partials<KL>(fake, 32, sc, am);
         if (lane == 0) { s_rehearsal[0] = sc; s_rehearsal[1] = __int_as_float(am); }
-        decide_sequence_rehearsal(p, &s_decide);
         for (int b = blockIdx.x; b < p.B; b += gridDim.x)
-            if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_decide);
+            if (count_flagged(p, b) == 0) decide_sequence(p, b, &s_no_area);
         // the scan's result
         int seen = 0;
         for (unsigned spin = 0; spin < (1u << 22); ++spin) {
@@ -192,6 +204,13 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
         } else {
             setup_lost = true;        // no range for this warp; reported below
         }
+        // The decision stage (only its register-resident forms: the general form for longer
+        // sequences is short loops written for a cold start, and a walk through it costs as much as
+        // the decision itself).  Where the launch has so little to stream (less than a unit for
+        // every other streaming warp of the grid) that its rows finish within microseconds, the
+        // walk is the short one: finished rows wait while this warp rehearses.
+        if (p.P <= 512)
+            decide_sequence_rehearsal(p, &s_decide, 2L * total_flagged * nch <= (long)kSConsumers * gridDim.x);
     }
     // equal ranges, each small enough for the table, their number a multiple of the CTAs
     const unsigned total_units = (unsigned)(total_flagged * nch);          // fits 31 bits (checked by the host)
@@ -490,7 +509,7 @@ __global__ void __launch_bounds__(kSThreads, 1) verify_stream_kernel(const Verif
                     const int b = __shfl_sync(full, e.row, from) / p.P;
                     const unsigned same = __ballot_sync(full, finished && e.row / p.P == b) & fin;
                     fin &= ~same;
-                    pending_add(p, pend, b, __popc(same), &s_decide);
+                    pending_add(p, pend, b, __popc(same), &s_no_area);
                 }
             }
         }

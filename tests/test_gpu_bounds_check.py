@@ -45,7 +45,7 @@ def both_builds(binding, check_path, call):
     (3, 40, 126464, 33, CONF),                   # the LLaDA vocabulary
     (2, 50, 1003, 31, KL),                       # V % 8 != 0: the element-wise kernel
     (15, 700, 64, 380, CONF | PROB),             # many short rows, sequences beyond the register-resident decision
-    (1, 1500, 4104, 900, TRUST | EMIT),          # a sequence beyond the staged decision
+    (1, 1500, 4104, 900, TRUST | EMIT),          # a sequence beyond the register-resident decision
     (4, 8, 8, 0, KL),                            # nothing flagged: every sequence passes through
 ])
 def test_verify_addresses_stay_inside(libs, B, P, V, flagged, mode):

@@ -82,10 +82,11 @@ def test_small_shapes_kl(dd, oracle_mod, B, P, K, V, flagged, mode):
             assert ref["out_mask"][fl].any() and not ref["out_mask"][fl].all()
 
 
-@pytest.mark.parametrize("P", [700, 1100])
+@pytest.mark.parametrize("P", [700, 1100, 2100])
 def test_long_sequences(dd, oracle_mod, P):
-    """Sequences longer than the register-resident decision stage holds (512 positions) and than
-    its staged form holds (1024): the fold kernel's deciding warp takes the general path."""
+    """Sequences longer than the register-resident decision stage holds (512 positions), longer
+    than the general form keeps in registers (1024), and longer than the fold kernel's key area in
+    shared memory (2048)."""
     hidden, weight, tokens, flags = synth.lm_head_inputs(2, P, 64, 520, "uniform_25_100", seed=P)
     compare(dd, oracle_mod, hidden, weight, tokens, flags, CONF | PROB, 0.05, 9, 11)
     dh, dw, vh, vw, tokens, flags = synth.lm_head_pair_inputs(2, P, 64, 520, "uniform_25_100", 0.2, seed=P + 1)

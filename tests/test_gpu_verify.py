@@ -141,13 +141,19 @@ def test_degenerate_cases(dd, oracle_mod):
 
 def test_many_short_rows_and_long_sequences(dd, oracle_mod):
     # more (row, chunk) units than the CTAs' tables hold at once (several rounds per CTA), and
-    # sequences longer than the decision stage keeps in shared memory
+    # sequences that exactly fill the decision stage's key area in shared memory (8192 keys)
     dra, ver, tokens, flags = synth.verify_inputs(15, 8192, 64, 5700, 0.2, seed=31)
     compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 40, 3)
     compare(dd, oracle_mod, dra, ver, tokens, flags, CONF | PROB, 0.5, 7, 3)
-    # a sequence length between the two decision paths' limits
+    # longer than what a lane keeps in registers (1024 keys), inside the key area
     dra, ver, tokens, flags = synth.verify_inputs(2, 1500, 4104, 900, 0.2, seed=32)
     compare(dd, oracle_mod, dra, ver, tokens, flags, KL, 0.5, 33, 1)
+    # the element-wise kernel (V % 8 != 0): inside its key area (2048 keys) and beyond it, where
+    # every pass of the decision stage re-reads the scores from memory (the streaming kernel's
+    # area holds the longest sequence the library accepts)
+    for P, nflag in ((1900, 1000), (2500, 1200)):
+        dra, ver, tokens, flags = synth.verify_inputs(1, P, 203, nflag, 0.2, seed=P)
+        compare(dd, oracle_mod, dra, ver, tokens, flags, KL | PROB, 0.5, 21, 5)
 
 
 def test_exact_ties_in_verifier_row(dd, oracle_mod):
