@@ -416,6 +416,10 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
         for nflag in synth.VERIFY_SWEEP["flagged"]:
             modes = (T, K_, C) if (V == 126464 and nflag == 512) else (K_,)
             ver_shapes.append((f"sweep V={V} masked={nflag}", 1, 512, V, nflag, 0.20, 8 if nflag == 32 else 32, modes))
+    # two shapes outside the configurations: a token excluded by both models (logit -inf at the same
+    # index in every row, e.g. the mask token) on the cfg1 shape, and a sequence of 1024 positions
+    ver_shapes.append(("cfg1 shape, one token excluded by both models", 1, 256, 126464, "all", 0.20, 32, (K_,)))
+    ver_shapes.append(("P=1024 V=32000 masked=128", 1, 1024, 32000, 128, 0.20, 32, (K_,)))
     mode_name = {T: "TRUST", K_: "KL", C: "CONF"}
     for name, B, P, V, flagged, err, k, modes in ver_shapes:
         want_d = K_ in modes
@@ -430,6 +434,10 @@ def other_configs(dd, stream, sampler, peaks, quick=False):
         if B * P * V * 2 > (1 << 30):
             ns = 1                                   # one set is already many times the L2
         sets = [device_logits(B, P, V, err, gen, want_d) for _ in range(ns)]
+        if "excluded" in name:
+            for dra, ver in sets:
+                dra[..., V - 128] = float("-inf")
+                ver[..., V - 128] = float("-inf")
         tokens = torch.randint(0, V, (B, P), device=dev, dtype=torch.int32, generator=gen)
         ot = torch.empty(B, P, device=dev, dtype=torch.int32)
         om = torch.empty(B, P, device=dev, dtype=torch.uint8)
