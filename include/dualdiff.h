@@ -94,6 +94,12 @@ int dd_bidir_attention(const void *q, const void *k, const void *v, void *out,
  *   out_score[b,i]  = KL_i (KL mode) or c_i (CONF and TRUST modes)
  * Positions with mask_flags == 0 pass through: out_tokens = tokens,
  * out_mask = 0, out_score = 0, and their logits are never read.
+ * A logit of -inf is an excluded token (probability 0, an ordinary input: a banned or
+ * padded vocabulary entry, the mask token): it contributes no term to Eq. 5 where the
+ * drafter excludes it (the sum runs over the support of p_D), and KL_i = +inf where
+ * only the verifier does.  In the streaming path that last case is recognised as long
+ * as the drafter gives the token at least 3e-35 of the probability mass of its stretch
+ * of 4096-8192 logits; below that the token counts as excluded by both.
  *
  * drafter_logits, verifier_logits: [B,P,V] bf16 (drafter_logits may be NULL
  * unless the mode is KL); tokens int32 [B,P]; mask_flags uint8 [B,P];
